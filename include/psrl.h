@@ -1,0 +1,207 @@
+/*
+ * psrl.h - C ABI of the tree-causal prefix-shared attention library (libpsrl.so).
+ *
+ * The library implements the attention step of training-time prefix sharing:
+ * samples of a step-wise or tree-structured RL batch share decision prefixes;
+ * every shared token span ("segment") is stored once, its K/V in a paged KV
+ * store, and each token attends to all tokens of its ancestor segments plus
+ * the causal part of its own segment, which reproduces per-sequence causal
+ * attention exactly (paper Sec. 2.5, "Prefix sharing in training").  Backward
+ * accumulates the adjoints of every consumer on the shared K/V (paper Sec. 6,
+ * "Prefix-sharing training runtime") in a fixed order, so results are bitwise
+ * reproducible run to run.
+ *
+ * Conventions
+ *  - Every call returns a psrl_status_t; nothing throws, aborts or prints.
+ *  - "host" / "device" is stated for every pointer.  The library never
+ *    allocates device memory in the entry points below: tensors, pools, the
+ *    plan's device mirror and the workspace are the caller's.
+ *  - Kernels are launched on the caller's stream; no entry point synchronises
+ *    except psrl_device_status().
+ *  - Only sm_100a devices are supported; there is no CPU or other fallback.
+ */
+#ifndef PSRL_H_
+#define PSRL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PSRL_OK = 0,
+  PSRL_ERR_INVALID_ARG = 1,    /* null / misaligned pointer, bad count, bad flag bits */
+  PSRL_ERR_BAD_TREE = 2,       /* parent >= own index, length < 1, leaf that ends no sample */
+  PSRL_ERR_BAD_BLOCK_SIZE = 3, /* block size not a power of two in [16, 256] */
+  PSRL_ERR_SHAPE = 4,          /* head counts do not divide, pool smaller than the plan needs */
+  PSRL_ERR_UNSUPPORTED = 5,    /* dtype x head_dim outside {f32 x {64,128}, bf16 x 128} */
+  PSRL_ERR_POOL_FULL = 6,      /* no free extent fits a page */
+  PSRL_ERR_WORKSPACE = 7,      /* workspace / device buffer too small, or plan not uploaded */
+  PSRL_ERR_HOST_OOM = 8,
+  PSRL_ERR_CUDA = 9,           /* a CUDA runtime / driver call failed */
+  PSRL_ERR_TIMEOUT = 10,       /* a bounded device-side wait ran out (read via psrl_device_status) */
+  PSRL_ERR_INTERNAL = 11
+} psrl_status_t;
+
+typedef enum { PSRL_F32 = 0, PSRL_BF16 = 1 } psrl_dtype_t;
+
+/* Segment flags. */
+enum {
+  PSRL_SEG_HAS_Q = 1,     /* the segment's tokens issue queries (rows of Q/O/dO/dQ exist) */
+  PSRL_SEG_SAMPLE_END = 2 /* a training sample ends at this segment (root-to-here path) */
+};
+
+/*
+ * Problem statement: a forest of token segments.  A sample is the path from a
+ * root to a SAMPLE_END segment (tree sampling: leaves; step / tree-step
+ * sampling: every node - paper Sec. 2.3).  Roots are independent prefix groups
+ * (paper Sec. 4.2, semantic groups).  All pointers are HOST pointers, read
+ * during psrl_plan_build only.
+ */
+typedef struct {
+  int32_t n_segments;              /* >= 1 */
+  const int32_t* parent;           /* [n_segments] -1 = root, else an index < own index */
+  const int32_t* seg_len;          /* [n_segments] tokens, >= 1 */
+  const uint8_t* seg_flags;        /* [n_segments] or NULL = HAS_Q everywhere, SAMPLE_END on leaves */
+  const int32_t* group_block_size; /* one per root, in input order; power of two in [16, 256] */
+  int32_t n_groups;                /* must equal the number of roots */
+  int32_t n_q_heads, n_kv_heads;   /* n_q_heads % n_kv_heads == 0 */
+  int32_t head_dim;                /* 64 or 128 (f32), 128 (bf16) */
+  psrl_dtype_t dtype;
+  const int32_t* free_extents;     /* [2 * n_free] (start_slot, n_slots), multiples of 16; NULL = bump from 0 */
+  int32_t n_free;
+} psrl_tree_desc_t;
+
+typedef struct psrl_plan psrl_plan_t;
+
+/*
+ * Borrowed HOST pointers into the plan's canonical arrays (valid until
+ * psrl_plan_destroy).  Segments are indexed in canonical order = DFS preorder,
+ * roots and siblings in ascending input index.  The per-page fields are the
+ * block metadata of the paper's KV manager (Sec. 6: base address, block size,
+ * position of the token span in the full sequence, reference count); pages
+ * follow reusable prefix spans and never cross a segment boundary (Sec. 5.1).
+ */
+typedef struct {
+  int32_t n_seg, n_groups, n_pages, n_samples, max_depth;
+  int32_t T;          /* tokens stored (each shared token once) */
+  int32_t T_q;        /* tokens that issue queries */
+  int32_t pool_slots; /* slots per KV head the pools must hold: max(page_slot + page_bs) */
+  int64_t flat_tokens; /* sum of sample lengths (the unshared layout) */
+  int64_t tree_pairs;  /* attended (query, key) pairs, shared:   sum len*anc + len(len+1)/2  (cf. Eq. 1) */
+  int64_t flat_pairs;  /* attended pairs, unshared: sum L(L+1)/2 */
+  int32_t n_anc, n_bt; /* lengths of anc_list and bt_pages */
+  const int32_t *canon_of_input, *input_of_canon;               /* [n_seg] */
+  const int32_t *seg_group, *seg_bs, *seg_parent, *seg_len, *seg_flags, *seg_depth;
+  const int32_t *seg_anc_tokens; /* tokens of strict ancestors = position of the span in the sequence */
+  const int32_t *seg_sub_end;    /* subtree = canonical indices [c, seg_sub_end[c]) */
+  const int32_t *seg_tok_off;    /* exclusive prefix sum of seg_len */
+  const int32_t *seg_q_off;      /* first row in Q/O/dO/dQ, -1 if the segment has no queries */
+  const int32_t *seg_refcount;   /* samples that pass through the segment (Sec. 5.2) */
+  const int32_t *anc_off, *anc_list;         /* CSR: strict ancestors root -> parent */
+  const int32_t *seg_first_page, *seg_n_pages;
+  const int32_t *page_seg, *page_bs, *page_valid, *page_pos, *page_refcount, *page_slot; /* [n_pages] */
+  const int32_t *bt_off, *bt_pages;          /* CSR block table: ancestors' pages root -> parent, then own */
+  const int32_t *tok_slot;                   /* [T] slot of every token in the pools */
+  const int32_t *sample_end_seg, *sample_len; /* [n_samples] */
+} psrl_plan_view_t;
+
+/*
+ * psrl_plan_build - host-side plan builder (paper Sec. 5.1 Adaptive Block
+ * Allocation, Sec. 5.2 reference counts, Sec. 6 block metadata).
+ * Turns the forest into the canonical plan (paged block table with a block
+ * size per group) and a device work schedule.  Pure host code, no CUDA call.
+ *   desc      HOST, read only during the call
+ *   out_plan  HOST, receives a plan owned by the library (psrl_plan_destroy)
+ * Errors: INVALID_ARG, BAD_TREE, BAD_BLOCK_SIZE, SHAPE, UNSUPPORTED,
+ * POOL_FULL, HOST_OOM.  On error *out_plan is NULL.
+ */
+psrl_status_t psrl_plan_build(const psrl_tree_desc_t* desc, psrl_plan_t** out_plan);
+
+/* Fills *out with borrowed host pointers.  INVALID_ARG on NULL. */
+psrl_status_t psrl_plan_view(const psrl_plan_t* plan, psrl_plan_view_t* out);
+
+/* Bytes of DEVICE memory psrl_plan_upload needs (0 for a NULL plan). */
+size_t psrl_plan_device_bytes(const psrl_plan_t* plan);
+
+/*
+ * Copies the device schedule into caller-owned DEVICE memory (256-byte
+ * aligned, >= psrl_plan_device_bytes) with cudaMemcpyAsync on `stream`
+ * (a cudaStream_t passed as void*; NULL = default stream) and binds the plan
+ * to that buffer.  The buffer must outlive every launch that uses the plan.
+ * Errors: INVALID_ARG, WORKSPACE (too small), CUDA.
+ */
+psrl_status_t psrl_plan_upload(psrl_plan_t* plan, void* dev_buf, size_t bytes, void* stream);
+
+/* Bytes of DEVICE workspace the forward / backward call needs (>= 256). */
+size_t psrl_fwd_workspace_bytes(const psrl_plan_t* plan);
+size_t psrl_bwd_workspace_bytes(const psrl_plan_t* plan);
+
+/*
+ * psrl_tree_attn_fwd - tree-causal attention forward (paper Sec. 2.5 attention
+ * masking; Sec. 6: the attention backend locates K/V through block metadata).
+ * For every query row i of a HAS_Q segment c and query head h (KV head
+ * h / (Hq/Hkv)):  keys = all tokens of c's ancestors + tokens 0..i of c;
+ *   O_i = softmax_j(scale * q_i . k_j) V,   LSE_i = ln sum_j exp(scale * q_i . k_j).
+ * All tensor pointers are DEVICE pointers, 16-byte aligned, dtype = plan dtype:
+ *   q        [T_q, Hq, d]  read only; rows of segment c start at seg_q_off[c]
+ *   k_pool   [Hkv, pool_capacity, d] read only; token t lives at slot tok_slot[t]
+ *   v_pool   same layout.  Slots that hold no token (page pads, free slots)
+ *            may contain anything, NaN included; they never reach an output.
+ *   pool_capacity  slots per KV head in the caller's pools, >= plan pool_slots
+ *   o        [T_q, Hq, d]  fully overwritten
+ *   lse      [Hq, T_q] fp32 fully overwritten (natural log, scale inside)
+ *   workspace, workspace_bytes  >= psrl_fwd_workspace_bytes(plan), 256-byte
+ *            aligned; holds the device status word.  Concurrent launches need
+ *            distinct workspaces.
+ *   stream   cudaStream_t as void*
+ * Errors: INVALID_ARG, SHAPE, WORKSPACE, CUDA.  Asynchronous.
+ */
+psrl_status_t psrl_tree_attn_fwd(const psrl_plan_t* plan, const void* q, const void* k_pool, const void* v_pool,
+                                 int64_t pool_capacity, void* o, float* lse, float softmax_scale,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * psrl_tree_attn_bwd - backward of the above (paper Sec. 6: consumer adjoints
+ * are accumulated on the shared prefix before one backward pass through its
+ * producer).  Given dO (one row per shared token, already summed over the
+ * samples that contain it):
+ *   P = exp(S - LSE), dV = P^T dO, dP = dO V^T, D_i = dO_i . O_i,
+ *   dS = P o (dP - D), dQ = scale dS K, dK = scale dS^T Q,
+ * where dK/dV of a token sum over every query row that attends to it (its own
+ * segment's later rows and all rows of all descendant segments) and over the
+ * Hq/Hkv query heads of its KV head, in a fixed order.
+ * DEVICE pointers, 16-byte aligned:
+ *   q, k_pool, v_pool, o, lse   as in / as produced by the forward; read only
+ *   d_o      [T_q, Hq, d] read only
+ *   d_q      [T_q, Hq, d] fully overwritten
+ *   dk_pool, dv_pool [Hkv, pool_capacity, d]: every slot of every page of the
+ *            plan is overwritten (token slots: gradient; pad slots: 0); slots
+ *            outside the plan's pages are not touched
+ *   workspace >= psrl_bwd_workspace_bytes(plan): status word + D [Hq, T_q] fp32
+ * Errors: INVALID_ARG, SHAPE, WORKSPACE, CUDA.  Asynchronous.
+ */
+psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const void* k_pool, const void* v_pool,
+                                 int64_t pool_capacity, const void* o, const float* lse, const void* d_o,
+                                 void* d_q, void* dk_pool, void* dv_pool, float softmax_scale, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+
+/*
+ * Synchronises `stream`, then reads the status word the last launch that used
+ * `workspace` left: PSRL_OK, PSRL_ERR_TIMEOUT (a bounded wait gave up; outputs
+ * are invalid) or PSRL_ERR_INTERNAL.  CUDA errors map to PSRL_ERR_CUDA.
+ */
+psrl_status_t psrl_device_status(const void* workspace, void* stream);
+
+/* Last CUDA error string seen by the library on this thread (HOST, static storage). */
+const char* psrl_last_cuda_error(void);
+
+void psrl_plan_destroy(psrl_plan_t* plan);
+const char* psrl_status_string(psrl_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSRL_H_ */

@@ -1,0 +1,320 @@
+"""ctypes binding of libpsrl.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs inside the library's kernels.  The binding raises
+if the library has not been built; there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpsrl.so")
+
+PSRL_OK = 0
+STATUS_NAMES = [
+    "PSRL_OK", "PSRL_ERR_INVALID_ARG", "PSRL_ERR_BAD_TREE", "PSRL_ERR_BAD_BLOCK_SIZE", "PSRL_ERR_SHAPE",
+    "PSRL_ERR_UNSUPPORTED", "PSRL_ERR_POOL_FULL", "PSRL_ERR_WORKSPACE", "PSRL_ERR_HOST_OOM", "PSRL_ERR_CUDA",
+    "PSRL_ERR_TIMEOUT", "PSRL_ERR_INTERNAL",
+]
+PSRL_F32, PSRL_BF16 = 0, 1
+SEG_HAS_Q, SEG_SAMPLE_END = 1, 2
+
+EXPORTS = [
+    "psrl_plan_build", "psrl_plan_view", "psrl_plan_device_bytes", "psrl_plan_upload",
+    "psrl_fwd_workspace_bytes", "psrl_bwd_workspace_bytes", "psrl_tree_attn_fwd", "psrl_tree_attn_bwd",
+    "psrl_device_status", "psrl_last_cuda_error", "psrl_plan_destroy", "psrl_status_string",
+]
+
+_I32P = C.POINTER(C.c_int32)
+
+
+class TreeDesc(C.Structure):
+    _fields_ = [
+        ("n_segments", C.c_int32), ("parent", _I32P), ("seg_len", _I32P), ("seg_flags", C.POINTER(C.c_uint8)),
+        ("group_block_size", _I32P), ("n_groups", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("dtype", C.c_int), ("free_extents", _I32P), ("n_free", C.c_int32),
+    ]
+
+
+_VIEW_SCALARS32 = ["n_seg", "n_groups", "n_pages", "n_samples", "max_depth", "T", "T_q", "pool_slots"]
+_VIEW_SCALARS64 = ["flat_tokens", "tree_pairs", "flat_pairs"]
+_VIEW_ARRAYS = [
+    "canon_of_input", "input_of_canon", "seg_group", "seg_bs", "seg_parent", "seg_len", "seg_flags", "seg_depth",
+    "seg_anc_tokens", "seg_sub_end", "seg_tok_off", "seg_q_off", "seg_refcount", "anc_off", "anc_list",
+    "seg_first_page", "seg_n_pages", "page_seg", "page_bs", "page_valid", "page_pos", "page_refcount", "page_slot",
+    "bt_off", "bt_pages", "tok_slot", "sample_end_seg", "sample_len",
+]
+
+
+class PlanView(C.Structure):
+    _fields_ = (
+        [(n, C.c_int32) for n in _VIEW_SCALARS32]
+        + [(n, C.c_int64) for n in _VIEW_SCALARS64]
+        + [("n_anc", C.c_int32), ("n_bt", C.c_int32)]
+        + [(n, _I32P) for n in _VIEW_ARRAYS]
+    )
+
+
+class PsrlError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where}: {name}{(' (' + detail + ')') if detail else ''}")
+        self.status = status
+        self.name = name
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libpsrl.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2608_25683_b200.build` "
+            "(there is no fallback path)")
+    L = C.CDLL(LIB_PATH)
+    L.psrl_plan_build.argtypes = [C.POINTER(TreeDesc), C.POINTER(C.c_void_p)]
+    L.psrl_plan_build.restype = C.c_int
+    L.psrl_plan_view.argtypes = [C.c_void_p, C.POINTER(PlanView)]
+    L.psrl_plan_view.restype = C.c_int
+    L.psrl_plan_device_bytes.argtypes = [C.c_void_p]
+    L.psrl_plan_device_bytes.restype = C.c_size_t
+    L.psrl_plan_upload.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    L.psrl_plan_upload.restype = C.c_int
+    for f in (L.psrl_fwd_workspace_bytes, L.psrl_bwd_workspace_bytes):
+        f.argtypes = [C.c_void_p]
+        f.restype = C.c_size_t
+    L.psrl_tree_attn_fwd.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                     C.c_void_p, C.c_float, C.c_void_p, C.c_size_t, C.c_void_p]
+    L.psrl_tree_attn_fwd.restype = C.c_int
+    L.psrl_tree_attn_bwd.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
+                                     C.c_void_p, C.c_size_t, C.c_void_p]
+    L.psrl_tree_attn_bwd.restype = C.c_int
+    L.psrl_device_status.argtypes = [C.c_void_p, C.c_void_p]
+    L.psrl_device_status.restype = C.c_int
+    L.psrl_last_cuda_error.restype = C.c_char_p
+    L.psrl_plan_destroy.argtypes = [C.c_void_p]
+    L.psrl_plan_destroy.restype = None
+    L.psrl_status_string.argtypes = [C.c_int]
+    L.psrl_status_string.restype = C.c_char_p
+    _lib = L
+    return L
+
+
+def _check(status: int, where: str):
+    if status != PSRL_OK:
+        detail = ""
+        if status == 9:
+            detail = lib().psrl_last_cuda_error().decode()
+        raise PsrlError(status, where, detail)
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+class Plan:
+    """Owner of a psrl_plan_t.  `view` holds numpy copies of the canonical arrays."""
+
+    def __init__(self, parent: Sequence[int], seg_len: Sequence[int], group_block_size: Sequence[int],
+                 n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: str,
+                 seg_flags: Optional[Sequence[int]] = None, free_extents=None):
+        self._h = C.c_void_p()
+        self._dev = None
+        self._ws = {}
+        L = lib()
+        p, l, g = _i32(parent), _i32(seg_len), _i32(group_block_size)
+        d = TreeDesc()
+        d.n_segments = len(p)
+        d.parent = p.ctypes.data_as(_I32P)
+        d.seg_len = l.ctypes.data_as(_I32P)
+        fl = None
+        if seg_flags is not None:
+            fl = np.ascontiguousarray(np.asarray(seg_flags, dtype=np.uint8))
+            d.seg_flags = fl.ctypes.data_as(C.POINTER(C.c_uint8))
+        d.group_block_size = g.ctypes.data_as(_I32P)
+        d.n_groups = len(g)
+        d.n_q_heads, d.n_kv_heads, d.head_dim = int(n_q_heads), int(n_kv_heads), int(head_dim)
+        d.dtype = {"f32": PSRL_F32, "bf16": PSRL_BF16}.get(dtype, 99)
+        fe = None
+        if free_extents is not None:
+            fe = _i32(np.asarray(free_extents, dtype=np.int64).reshape(-1))
+            d.free_extents = fe.ctypes.data_as(_I32P)
+            d.n_free = len(fe) // 2
+        _check(L.psrl_plan_build(C.byref(d), C.byref(self._h)), "psrl_plan_build")
+        self.n_q_heads, self.n_kv_heads, self.head_dim, self.dtype = int(n_q_heads), int(n_kv_heads), int(head_dim), dtype
+        v = PlanView()
+        _check(L.psrl_plan_view(self._h, C.byref(v)), "psrl_plan_view")
+        self.view = self._copy_view(v)
+
+    @staticmethod
+    def _copy_view(v: PlanView) -> dict:
+        out = {n: int(getattr(v, n)) for n in _VIEW_SCALARS32 + _VIEW_SCALARS64}
+        n_seg, n_pages = out["n_seg"], out["n_pages"]
+        sizes = {n: n_seg for n in _VIEW_ARRAYS}
+        sizes.update(anc_off=n_seg + 1, anc_list=int(v.n_anc), bt_off=n_seg + 1, bt_pages=int(v.n_bt),
+                     tok_slot=out["T"], sample_end_seg=out["n_samples"], sample_len=out["n_samples"])
+        for n in ("page_seg", "page_bs", "page_valid", "page_pos", "page_refcount", "page_slot"):
+            sizes[n] = n_pages
+        for n in _VIEW_ARRAYS:
+            sz = sizes[n]
+            ptr = getattr(v, n)
+            out[n] = np.ctypeslib.as_array(ptr, shape=(sz,)).copy() if sz > 0 else np.zeros(0, dtype=np.int32)
+        return out
+
+    @property
+    def handle(self):
+        return self._h
+
+    def device_bytes(self) -> int:
+        return int(lib().psrl_plan_device_bytes(self._h))
+
+    def fwd_workspace_bytes(self) -> int:
+        return int(lib().psrl_fwd_workspace_bytes(self._h))
+
+    def bwd_workspace_bytes(self) -> int:
+        return int(lib().psrl_bwd_workspace_bytes(self._h))
+
+    def upload(self, device="cuda", stream=None):
+        """Allocate the device mirror with torch and upload the schedule."""
+        import torch
+
+        buf = torch.empty(self.device_bytes() + 256, dtype=torch.uint8, device=device)
+        ptr = (buf.data_ptr() + 255) // 256 * 256
+        s = _stream_ptr(stream)
+        _check(lib().psrl_plan_upload(self._h, C.c_void_p(ptr), self.device_bytes(), s), "psrl_plan_upload")
+        self._dev = buf
+        return self
+
+    def workspace(self, kind: str, device="cuda"):
+        """A cached torch workspace of the right size ('fwd' | 'bwd'); returns (ptr, bytes)."""
+        import torch
+
+        need = self.fwd_workspace_bytes() if kind == "fwd" else self.bwd_workspace_bytes()
+        key = (kind, str(device))
+        if key not in self._ws:
+            self._ws[key] = torch.empty(need + 256, dtype=torch.uint8, device=device)
+        buf = self._ws[key]
+        return (buf.data_ptr() + 255) // 256 * 256, need
+
+    def close(self):
+        if self._h:
+            lib().psrl_plan_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def _stream_ptr(stream) -> C.c_void_p:
+    if stream is None:
+        import torch
+
+        if torch.cuda.is_available():
+            return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+        return C.c_void_p(0)
+    if hasattr(stream, "cuda_stream"):
+        return C.c_void_p(stream.cuda_stream)
+    return C.c_void_p(int(stream))
+
+
+def psrl_tree_attn_fwd(plan: Plan, q, k_pool, v_pool, softmax_scale: float, o=None, lse=None, stream=None,
+                       workspace=None):
+    """Forward.  q [T_q,Hq,d], pools [Hkv,capacity,d] torch CUDA tensors of the
+    plan's dtype.  Returns (o, lse); both are allocated with torch if not given."""
+    import torch
+
+    V = plan.view
+    assert q.is_contiguous() and k_pool.is_contiguous() and v_pool.is_contiguous()
+    assert tuple(q.shape) == (V["T_q"], plan.n_q_heads, plan.head_dim), q.shape
+    assert k_pool.shape == v_pool.shape and k_pool.shape[0] == plan.n_kv_heads and k_pool.shape[2] == plan.head_dim
+    _check_dtype(plan, q, k_pool, v_pool)
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((plan.n_q_heads, V["T_q"]), dtype=torch.float32, device=q.device)
+    ws, wsb = workspace if workspace is not None else plan.workspace("fwd", q.device)
+    st = lib().psrl_tree_attn_fwd(plan.handle, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(),
+                                  int(k_pool.shape[1]), o.data_ptr(), lse.data_ptr(), float(softmax_scale),
+                                  C.c_void_p(ws), wsb, _stream_ptr(stream))
+    _check(st, "psrl_tree_attn_fwd")
+    return o, lse
+
+
+def psrl_tree_attn_bwd(plan: Plan, q, k_pool, v_pool, o, lse, d_o, softmax_scale: float, d_q=None, dk_pool=None,
+                       dv_pool=None, stream=None, workspace=None):
+    """Backward.  Returns (d_q, dk_pool, dv_pool).  dk/dv pools are allocated
+    zero-filled if not given (the library itself only writes the plan's pages)."""
+    import torch
+
+    _check_dtype(plan, q, k_pool, v_pool, o, d_o)
+    assert d_o.is_contiguous() and o.is_contiguous() and lse.is_contiguous()
+    if d_q is None:
+        d_q = torch.empty_like(q)
+    if dk_pool is None:
+        dk_pool = torch.zeros_like(k_pool)
+    if dv_pool is None:
+        dv_pool = torch.zeros_like(v_pool)
+    ws, wsb = workspace if workspace is not None else plan.workspace("bwd", q.device)
+    st = lib().psrl_tree_attn_bwd(plan.handle, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(),
+                                  int(k_pool.shape[1]), o.data_ptr(), lse.data_ptr(), d_o.data_ptr(), d_q.data_ptr(),
+                                  dk_pool.data_ptr(), dv_pool.data_ptr(), float(softmax_scale), C.c_void_p(ws), wsb,
+                                  _stream_ptr(stream))
+    _check(st, "psrl_tree_attn_bwd")
+    return d_q, dk_pool, dv_pool
+
+
+def psrl_device_status(plan: Plan, kind: str = "fwd", stream=None, device="cuda") -> int:
+    ws, _ = plan.workspace(kind, device)
+    return int(lib().psrl_device_status(C.c_void_p(ws), _stream_ptr(stream)))
+
+
+def _check_dtype(plan: Plan, *tensors):
+    import torch
+
+    want = torch.float32 if plan.dtype == "f32" else torch.bfloat16
+    for t in tensors:
+        if t.dtype != want:
+            raise TypeError(f"tensor dtype {t.dtype} does not match the plan's {want}")
+        if not t.is_cuda:
+            raise RuntimeError("tensors must live on a CUDA device: this library has no CPU path")
+
+
+def flatten_forest(view: dict):
+    """The unshared layout: every sample becomes a root segment of its own
+    holding copies of its tokens (what a system without prefix sharing stores).
+
+    Returns (parent, seg_len, group_block_size, tok_src, first_copy) where
+    tok_src[i] is the tree token copied to flat token i and first_copy[i] says
+    whether it is that token's first copy in canonical sample order (the copy
+    that carries the token's upstream gradient row; the others get zero).
+    """
+    parent, seg_len, gbs, src = [], [], [], []
+    for e in view["sample_end_seg"]:
+        e = int(e)
+        path = list(view["anc_list"][view["anc_off"][e]:view["anc_off"][e + 1]]) + [e]
+        L = 0
+        for c in path:
+            t0 = int(view["seg_tok_off"][c])
+            n = int(view["seg_len"][c])
+            src.append(np.arange(t0, t0 + n, dtype=np.int64))
+            L += n
+        parent.append(-1)
+        seg_len.append(L)
+        gbs.append(int(view["seg_bs"][e]))
+    tok_src = np.concatenate(src)
+    _, first_idx = np.unique(tok_src, return_index=True)
+    first_copy = np.zeros(len(tok_src), dtype=bool)
+    first_copy[first_idx] = True
+    return parent, seg_len, gbs, tok_src, first_copy

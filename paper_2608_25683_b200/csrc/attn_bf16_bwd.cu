@@ -1,0 +1,4 @@
+#include "kernels.h"
+namespace psrl {
+psrl_status_t bwd_bf16(const AttnArgs&) { return PSRL_ERR_UNSUPPORTED; }
+}

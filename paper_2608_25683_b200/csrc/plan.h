@@ -1,0 +1,84 @@
+// Internal representation of a plan: the canonical arrays the C ABI exposes
+// through psrl_plan_view_t plus the device work schedule the kernels consume.
+#pragma once
+#include <cstdint>
+#include <vector>
+
+#include "../../include/psrl.h"
+
+namespace psrl {
+
+constexpr int kTile = 128;  // rows of a query tile / keys of a KV tile on the tensor-core path
+
+// One KV tile: up to 128 consecutive tokens of ONE segment (tiles never cross
+// a segment boundary, so the valid rows are always a prefix of the tile).
+struct KvTile {
+  int32_t first_page;  // first page of the tile
+  int32_t n_pages;     // pages the tile spans (1 when bs >= 128)
+  int32_t bs;          // page size of the segment's group
+  int32_t row_off;     // first row inside first_page (0, or 128 for the upper half of a 256-slot page)
+  int32_t n_valid;     // valid keys in the tile (1..128)
+  int32_t seg;         // canonical segment
+  int32_t tile_idx;    // index of the tile inside its segment
+  int32_t rows_loaded; // rows a gather brings in: n_pages * min(bs, 128)
+};
+
+// One query tile: up to 128 consecutive rows of one HAS_Q segment.
+struct QTile {
+  int32_t seg;
+  int32_t tile_idx;   // rows [tile_idx*128, ...) of the segment
+  int32_t q_row0;     // first row in Q/O/dO/dQ
+  int32_t n_rows;     // 1..128
+  int32_t pt_begin;   // range in path_tiles: ancestors' tiles root->parent, then own tiles 0..tile_idx
+  int32_t n_kv_tiles; // tiles to visit; the last one is the diagonal tile
+  int32_t pad0, pad1;
+};
+
+// One dK/dV work item: a KV tile and the query rows that attend to it.
+struct KvItem {
+  int32_t kvt;         // KV tile id
+  int32_t own_q_row0;  // first own-segment query row (the tile's first key), -1 if the segment has no queries
+  int32_t own_q_end;   // one past the segment's last query row
+  int32_t desc_q_begin, desc_q_end;  // query rows of all strict descendants (contiguous), empty if none
+  int32_t pad0, pad1, pad2;
+};
+
+// Offsets (in int32 units from the start of the device blob) of each array.
+struct DeviceHeader {
+  int32_t magic;
+  int32_t n_seg, n_pages, n_kvt, n_qt, T, T_q, n_bt;
+  int32_t off_seg_len, off_seg_q_off, off_seg_tok_off, off_seg_flags, off_seg_first_page, off_seg_n_pages;
+  int32_t off_seg_bs, off_seg_first_kvt, off_seg_n_kvt, off_seg_desc_q_begin, off_seg_desc_q_end;
+  int32_t off_page_slot, off_page_valid, off_page_seg, off_page_bs;
+  int32_t off_bt_off, off_bt_pages;
+  int32_t off_qrow_seg;  // [T_q] segment of every query row
+  int32_t off_kvt, off_qt, off_kvi, off_path_off, off_path_tiles;
+  int32_t reserved[8];
+};
+
+struct Plan {
+  // problem
+  int32_t Hq = 0, Hkv = 0, d = 0;
+  psrl_dtype_t dtype = PSRL_F32;
+  // scalars
+  int32_t n_seg = 0, n_groups = 0, n_pages = 0, n_samples = 0, max_depth = 0, T = 0, T_q = 0, pool_slots = 0;
+  int64_t flat_tokens = 0, tree_pairs = 0, flat_pairs = 0;
+  // canonical arrays
+  std::vector<int32_t> canon_of_input, input_of_canon, seg_group, seg_bs, seg_parent, seg_len, seg_flags, seg_depth,
+      seg_anc_tokens, seg_sub_end, seg_tok_off, seg_q_off, seg_refcount, anc_off, anc_list, seg_first_page,
+      seg_n_pages, page_seg, page_bs, page_valid, page_pos, page_refcount, page_slot, bt_off, bt_pages, tok_slot,
+      sample_end_seg, sample_len;
+  // schedule (host copies)
+  std::vector<KvTile> kv_tiles;
+  std::vector<QTile> q_tiles;    // longest first
+  std::vector<KvItem> kv_items;  // longest first
+  std::vector<int32_t> seg_first_kvt, seg_n_kvt, seg_desc_q_begin, seg_desc_q_end, path_off, path_tiles, qrow_seg;
+  // device blob
+  std::vector<int32_t> blob;
+  DeviceHeader hdr{};
+  const int32_t* dev = nullptr;  // bound device copy of blob
+};
+
+psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out);
+
+}  // namespace psrl
