@@ -199,7 +199,7 @@ class Plan:
         import torch
 
         need = self.fwd_workspace_bytes() if kind == "fwd" else self.bwd_workspace_bytes()
-        key = (kind, str(device))
+        key = (kind, str(torch.device(device if self._dev is None else self._dev.device)))
         if key not in self._ws:
             self._ws[key] = torch.empty(need + 256, dtype=torch.uint8, device=device)
         buf = self._ws[key]

@@ -1,6 +1,6 @@
 // fp32 SIMT tree attention, forward and backward.
 //
-// This is the exact-arithmetic path (fp32 inputs, fp32 FMA, max-abs 1e-5
+// This is the exact-arithmetic path (fp32 inputs, fp32 products, fp64 running sums, max-abs 1e-5
 // against the fp64 definition); tensor cores cannot meet that bound, so the
 // kernels are plain CUDA: one warp per (query row, query head) for the forward
 // and dQ, one warp per (key slot, KV head) for dK/dV.  Every output element is
@@ -90,11 +90,14 @@ row_kernel(DevPlan dp, int Hq, int G, int64_t cap, float scale, const float* __r
   const int c = dp.qrow_seg[r];
   const int i = r - dp.seg_q_off[c];
   const int first_page = dp.seg_first_page[c];
-  float qv[VEC], acc[VEC], dov[VEC];
+  // long sums are kept in fp64 so that the 1e-5 bound holds for thousands of keys
+  float qv[VEC], dov[VEC];
+  double acc[VEC];
   load_vec<VEC>(qv, q + (int64_t(r) * Hq + h) * D + lane * VEC);
 #pragma unroll
-  for (int x = 0; x < VEC; ++x) acc[x] = 0.f;
-  float m = -CUDART_INF_F, l = 0.f, lse = 0.f, dl = 0.f;
+  for (int x = 0; x < VEC; ++x) acc[x] = 0.0;
+  float m = -CUDART_INF_F, lse = 0.f, dl = 0.f;
+  double l = 0.0;
   if (MODE == 1) {
     load_vec<VEC>(dov, d_o + (int64_t(r) * Hq + h) * D + lane * VEC);
     lse = lse_in[int64_t(h) * dp.T_q + r];
@@ -120,9 +123,9 @@ row_kernel(DevPlan dp, int Hq, int G, int64_t cap, float scale, const float* __r
         const float m_new = fmaxf(m, s);
         const float alpha = expf(m - m_new);
         const float p = expf(s - m_new);
-        l = fmaf(l, alpha, p);
+        l = l * double(alpha) + double(p);
 #pragma unroll
-        for (int x = 0; x < VEC; ++x) acc[x] = fmaf(acc[x], alpha, p * vv[x]);
+        for (int x = 0; x < VEC; ++x) acc[x] = acc[x] * double(alpha) + double(p) * double(vv[x]);
         m = m_new;
       } else {
         float s = dot<VEC>(qv, kv), t = dot<VEC>(dov, vv);
@@ -134,20 +137,21 @@ row_kernel(DevPlan dp, int Hq, int G, int64_t cap, float scale, const float* __r
         const float p = expf(s * scale - lse);
         const float ds = p * (t - dl);
 #pragma unroll
-        for (int x = 0; x < VEC; ++x) acc[x] = fmaf(ds, kv[x], acc[x]);
+        for (int x = 0; x < VEC; ++x) acc[x] += double(ds) * double(kv[x]);
       }
     }
   }
   if (MODE == 0) {
-    const float inv = 1.f / l;
+    float out[VEC];
 #pragma unroll
-    for (int x = 0; x < VEC; ++x) acc[x] *= inv;
-    store_vec<VEC>(o_out + (int64_t(r) * Hq + h) * D + lane * VEC, acc);
-    if (lane == 0) lse_out[int64_t(h) * dp.T_q + r] = m + logf(l);
+    for (int x = 0; x < VEC; ++x) out[x] = float(acc[x] / l);
+    store_vec<VEC>(o_out + (int64_t(r) * Hq + h) * D + lane * VEC, out);
+    if (lane == 0) lse_out[int64_t(h) * dp.T_q + r] = float(double(m) + log(l));
   } else {
+    float out[VEC];
 #pragma unroll
-    for (int x = 0; x < VEC; ++x) acc[x] *= scale;
-    store_vec<VEC>(d_q + (int64_t(r) * Hq + h) * D + lane * VEC, acc);
+    for (int x = 0; x < VEC; ++x) out[x] = float(acc[x] * double(scale));
+    store_vec<VEC>(d_q + (int64_t(r) * Hq + h) * D + lane * VEC, out);
   }
 }
 
@@ -186,9 +190,9 @@ dkv_kernel(DevPlan dp, int Hq, int G, int64_t cap, float scale, const float* __r
   const int q_off = dp.seg_q_off[a], len = dp.seg_len[a];
   const int dqb = dp.seg_desc_q_begin[a], dqe = dp.seg_desc_q_end[a];
   for (int j = warp; j < bs; j += kWarpsPerBlock) {
-    float dk[VEC], dv[VEC];
+    double dk[VEC], dv[VEC];
 #pragma unroll
-    for (int x = 0; x < VEC; ++x) dk[x] = dv[x] = 0.f;
+    for (int x = 0; x < VEC; ++x) dk[x] = dv[x] = 0.0;
     const int64_t row = (int64_t(hk) * cap + slot0 + j) * D + lane * VEC;
     if (j < valid) {
       float kv[VEC], vv[VEC];
@@ -221,17 +225,21 @@ dkv_kernel(DevPlan dp, int Hq, int G, int64_t cap, float scale, const float* __r
             const float ds = p * (t - delta[int64_t(h) * dp.T_q + r]);
 #pragma unroll
             for (int x = 0; x < VEC; ++x) {
-              dv[x] = fmaf(p, dov[x], dv[x]);
-              dk[x] = fmaf(ds, qv[x], dk[x]);
+              dv[x] += double(p) * double(dov[x]);
+              dk[x] += double(ds) * double(qv[x]);
             }
           }
         }
       }
-#pragma unroll
-      for (int x = 0; x < VEC; ++x) dk[x] *= scale;
     }
-    store_vec<VEC>(dkp + row, dk);
-    store_vec<VEC>(dvp + row, dv);
+    float dko[VEC], dvo[VEC];
+#pragma unroll
+    for (int x = 0; x < VEC; ++x) {
+      dko[x] = float(dk[x] * double(scale));
+      dvo[x] = float(dv[x]);
+    }
+    store_vec<VEC>(dkp + row, dko);
+    store_vec<VEC>(dvp + row, dvo);
   }
 }
 
