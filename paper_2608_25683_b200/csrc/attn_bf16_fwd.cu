@@ -1,4 +1,345 @@
+// bf16 tree attention forward on the 5th-generation tensor cores.
+//
+// One CTA = one query tile (up to 128 rows of one segment) x up to two query
+// heads of the same KV head.  It walks the tile's path of KV tiles (all tiles
+// of the ancestor segments, then the own segment's tiles up to the diagonal;
+// paper Sec. 2.5: full visibility of the shared prefix + causal own suffix),
+// gathering K/V pages from the paged pools through the block metadata
+// (Sec. 6) with TMA.
+//
+// Warp roles (NQ = 2):
+//   warps 0-3   softmax warpgroup of head 0   (one query row per thread)
+//   warps 4-7   softmax warpgroup of head 1
+//   warp  8     TMA producer (Q once, then the K and V rings)
+//   warp  9     MMA issuer + TMEM owner
+// Tensor memory (512 columns): per head q, S_q at q*256 (128 fp32 columns,
+// later overwritten by P_q as packed bf16 in its first 64 columns) and the
+// per-tile product O_q = P_q V at q*256+128.
+//   S = Q K^T      tcgen05.mma, A and B from shared memory (K-major, 128B swizzle)
+//   O_tile = P V   tcgen05.mma, A = P from tensor memory, B = V (MN-major)
+// The MMA issuer alternates between the two heads, so the tensor cores work
+// on one head while the other head's warpgroup does its softmax.  Each softmax
+// thread keeps the running max / sum and the output row (128 fp32) in
+// registers; per-tile products are read back from tensor memory and folded in
+// with the rescale factor (online softmax; partial results merged by
+// log-sum-exp), so tensor memory never needs rescaling.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "attn_bf16_common.cuh"
 #include "kernels.h"
+#include "tma.h"
+
 namespace psrl {
-psrl_status_t fwd_bf16(const AttnArgs&) { return PSRL_ERR_UNSUPPORTED; }
+namespace {
+using namespace sm100;
+
+constexpr int NQ = 2;                    // query heads per CTA
+constexpr int KS = 2, VS = 2;            // K and V ring depths
+constexpr int kThreads = (4 * NQ + 2) * 32;
+
+struct FwdMaps {
+  CUtensorMap q;
+  PoolMaps kv;
+};
+
+struct FwdParams {
+  const int32_t* blob;
+  int32_t off_qt, off_kvt, off_path_tiles, off_path_nvalid, off_page_slot;
+  int32_t Hq, Hkv, G, T_q, pairs_per_group;
+  int64_t cap;
+  float scale_log2;
+  __nv_bfloat16* o;
+  float* lse;
+  int* status;
+};
+
+struct __align__(8) Barriers {
+  uint64_t q_full;
+  uint64_t k_full[KS], k_empty[KS], v_full[VS], v_empty[VS];
+  uint64_t s_full[NQ], p_ready[NQ], o_full[NQ], o_empty[NQ];
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;                          // NQ tiles
+  uint8_t* sK = sQ + NQ * kTileBytes;          // KS tiles
+  uint8_t* sV = sK + KS * kTileBytes;          // VS tiles
+  __shared__ Barriers bar;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // ---- which work item ----
+  const int units = p.Hkv * p.pairs_per_group;
+  const int item = blockIdx.x / units, u = blockIdx.x % units;
+  const int hk = u / p.pairs_per_group, pair = u % p.pairs_per_group;
+  const int h0 = hk * p.G + pair * NQ;
+  const int nq = min(NQ, p.G - pair * NQ);
+  const QTile qt = reinterpret_cast<const QTile*>(p.blob + p.off_qt)[item];
+  const int32_t* path_tiles = p.blob + p.off_path_tiles + qt.pt_begin;
+  const int32_t* path_nvalid = p.blob + p.off_path_nvalid + qt.pt_begin;
+  const int n_tiles = qt.n_kv_tiles;
+
+  if (tid == 0) {
+    s_abort = 0;
+    mbar_init(&bar.q_full, 1);
+    for (int i = 0; i < KS; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1); }
+    for (int i = 0; i < VS; ++i) { mbar_init(&bar.v_full[i], 1); mbar_init(&bar.v_empty[i], 1); }
+    for (int i = 0; i < NQ; ++i) {
+      mbar_init(&bar.s_full[i], 1); mbar_init(&bar.p_ready[i], 128);
+      mbar_init(&bar.o_full[i], 1); mbar_init(&bar.o_empty[i], 128);
+    }
+    fence_mbar_init();
+  }
+  if (warp == 4 * NQ + 1) { tmem_alloc(&s_tmem, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  volatile int* abortp = &s_abort;
+
+  if (warp == 4 * NQ) {
+    // ======================= TMA producer =======================
+    if (lane == 0) {
+      tma_prefetch_desc(&maps.q);
+      mbar_expect_tx(&bar.q_full, uint32_t(nq) * kTileBytes);
+      for (int q = 0; q < nq; ++q) {
+        load_row_tile(sQ + q * kTileBytes, &maps.q, &bar.q_full, h0 + q, qt.q_row0);
+      }
+      const KvTile* kvt = reinterpret_cast<const KvTile*>(p.blob + p.off_kvt);
+      const int32_t* page_slot = p.blob + p.off_page_slot;
+      const int64_t head_row0 = int64_t(hk) * p.cap;
+      for (int j = 0; j < n_tiles; ++j) {
+        const KvTile kt = kvt[path_tiles[j]];
+        const int ks = j % KS, vs = j % VS;
+        if (j >= KS && !mbar_wait(&bar.k_empty[ks], ((j / KS) + 1) & 1, abortp, p.status)) break;
+        load_kv_tile(sK + ks * kTileBytes, maps.kv.k, &bar.k_full[ks], kt, page_slot, head_row0);
+        if (j >= VS && !mbar_wait(&bar.v_empty[vs], ((j / VS) + 1) & 1, abortp, p.status)) break;
+        load_kv_tile(sV + vs * kTileBytes, maps.kv.v, &bar.v_full[vs], kt, page_slot, head_row0);
+      }
+    }
+  } else if (warp == 4 * NQ + 1) {
+    // ======================= MMA issuer =======================
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);   // S = Q K^T, both K-major
+      constexpr uint32_t idesc_o = make_idesc(128, 128, 0, 1);   // O = P V, V is MN-major
+      auto issue_s = [&](int q, int ks) {
+        const uint32_t a0 = smem_u32(sQ + q * kTileBytes), b0 = smem_u32(sK + ks * kTileBytes);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
+          mma_ss(tmem + q * 256, make_desc(a0 + off, 16, 1024), make_desc(b0 + off, 16, 1024), idesc_s, k > 0);
+        }
+      };
+      auto issue_pv = [&](int q, int vs) {
+        const uint32_t b0 = smem_u32(sV + vs * kTileBytes);
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          mma_ts(tmem + q * 256 + 128, tmem + q * 256 + k * 8, make_desc(b0 + k * 2048, kHalfBytes, 1024), idesc_o,
+                 k > 0);
+      };
+      bool ok = mbar_wait(&bar.q_full, 0, abortp, p.status) && mbar_wait(&bar.k_full[0], 0, abortp, p.status);
+      if (ok) {
+        tc_fence_after();
+        for (int q = 0; q < nq; ++q) { issue_s(q, 0); mma_commit(&bar.s_full[q]); }
+        mma_commit(&bar.k_empty[0]);
+      }
+      for (int j = 0; ok && j < n_tiles; ++j) {
+        const int vs = j % VS;
+        for (int q = 0; ok && q < nq; ++q) {
+          ok = mbar_wait(&bar.p_ready[q], j & 1, abortp, p.status);
+          if (ok && j > 0) ok = mbar_wait(&bar.o_empty[q], (j - 1) & 1, abortp, p.status);
+          if (ok && q == 0) ok = mbar_wait(&bar.v_full[vs], (j / VS) & 1, abortp, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(q, vs);
+          mma_commit(&bar.o_full[q]);
+          if (q == nq - 1) mma_commit(&bar.v_empty[vs]);
+          if (j + 1 < n_tiles) {
+            const int ks = (j + 1) % KS;
+            if (q == 0) ok = mbar_wait(&bar.k_full[ks], ((j + 1) / KS) & 1, abortp, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            issue_s(q, ks);
+            mma_commit(&bar.s_full[q]);
+            if (q == nq - 1) mma_commit(&bar.k_empty[ks]);
+          }
+        }
+      }
+    }
+  } else if (warp < 4 * nq) {
+    // ======================= softmax warpgroups =======================
+    const int q = warp >> 2;
+    const int row = tid & 127;                                  // query row inside the tile
+    const uint32_t t_lane = tmem + (uint32_t((warp & 3) * 32) << 16) + q * 256;
+    float acc[128];
+#pragma unroll
+    for (int i = 0; i < 128; ++i) acc[i] = 0.f;
+    float m_run = -CUDART_INF_F, l_run = 0.f, alpha_prev = 1.f;
+    bool ok = true;
+    int nv_next = path_nvalid[0];
+    for (int j = 0; j < n_tiles; ++j) {
+      const int n_valid = nv_next;
+      if (j + 1 < n_tiles) nv_next = path_nvalid[j + 1];
+      const bool diag = (j == n_tiles - 1);
+      const int limit = diag ? min(row + 1, n_valid) : n_valid;  // keys [0, limit) are visible
+      const bool need_mask = diag || n_valid < 128;
+      // ---- fold the previous tile's product into the running output ----
+      if (j > 0) {
+        ok = mbar_wait(&bar.o_full[q], (j - 1) & 1, abortp, p.status);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_lane + 128 + c * 32, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[c * 32 + i] = fmaf(acc[c * 32 + i], alpha_prev, __uint_as_float(r[i]));
+        }
+        tc_fence_before();
+        mbar_arrive(&bar.o_empty[q]);
+      }
+      // ---- softmax of this tile ----
+      ok = mbar_wait(&bar.s_full[q], j & 1, abortp, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      float mx = -CUDART_INF_F;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_lane + c * 32, r);
+        tmem_wait_ld();
+        if (need_mask) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (c * 32 + i < limit) ? __uint_as_float(r[i]) : -CUDART_INF_F);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+        }
+      }
+      const float m_new = fmaxf(m_run, mx * p.scale_log2);
+      // a row that sees no key yet keeps m = -inf; use 0 as the reference then so exp2 stays finite
+      const float m_ref = (m_new == -CUDART_INF_F) ? 0.f : m_new;
+      const float alpha = ex2(m_run - m_ref);
+      float sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32], pk[16];
+        tmem_ld32(t_lane + c * 32, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          float e0 = ex2(fmaf(__uint_as_float(r[i]), p.scale_log2, -m_ref));
+          float e1 = ex2(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, -m_ref));
+          if (need_mask) {
+            e0 = (c * 32 + i < limit) ? e0 : 0.f;
+            e1 = (c * 32 + i + 1 < limit) ? e1 : 0.f;
+          }
+          sum += e0 + e1;
+          pk[i >> 1] = pack_bf16(e0, e1);
+        }
+        tmem_st16(t_lane + c * 16, pk);
+      }
+      l_run = fmaf(l_run, alpha, sum);
+      m_run = m_new;
+      alpha_prev = alpha;
+      // V rows at or beyond n_valid (page pads, rows no page covers) must be zero before P V
+      if (q == 0 && n_valid < 128) {
+        ok = mbar_wait(&bar.v_full[j % VS], (j / VS) & 1, abortp, p.status);
+        if (!ok) break;
+        if (row >= n_valid) zero_tile_row(sV + (j % VS) * kTileBytes, row);
+        fence_proxy_async();
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bar.p_ready[q]);
+    }
+    // ---- last tile's product, normalise, store ----
+    if (ok) ok = mbar_wait(&bar.o_full[q], (n_tiles - 1) & 1, abortp, p.status);
+    if (ok) {
+      tc_fence_after();
+      const float inv = 1.f / l_run;
+      const bool store = row < qt.n_rows;
+      const int h = h0 + q;
+      __nv_bfloat16* orow = p.o + (int64_t(qt.q_row0 + row) * p.Hq + h) * 128;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_lane + 128 + c * 32, r);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float a0 = fmaf(acc[c * 32 + i], alpha_prev, __uint_as_float(r[i])) * inv;
+          const float a1 = fmaf(acc[c * 32 + i + 1], alpha_prev, __uint_as_float(r[i + 1])) * inv;
+          pk[i >> 1] = pack_bf16(a0, a1);
+        }
+        if (store) {
+#pragma unroll
+          for (int x = 0; x < 4; ++x)
+            *reinterpret_cast<uint4*>(orow + c * 32 + x * 8) = make_uint4(pk[4 * x], pk[4 * x + 1], pk[4 * x + 2], pk[4 * x + 3]);
+        }
+      }
+      if (store) p.lse[int64_t(h) * p.T_q + qt.q_row0 + row] = (m_run + log2f(l_run)) * kLn2;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4 * NQ + 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
 }
+
+}  // namespace
+
+bool make_pool_maps(PoolMaps* maps, const void* k_pool, const void* v_pool, int Hkv, int64_t cap) {
+  const uint32_t rows[4] = {16, 32, 64, 128};
+  for (int i = 0; i < 4; ++i) {
+    if (!make_map_bf16_2d(&maps->k[i], k_pool, 128, uint64_t(Hkv) * cap, 256, rows[i])) return false;
+    if (!make_map_bf16_2d(&maps->v[i], v_pool, 128, uint64_t(Hkv) * cap, 256, rows[i])) return false;
+  }
+  return true;
+}
+
+psrl_status_t fwd_bf16(const AttnArgs& a) {
+  const Plan& P = *a.plan;
+  const int64_t cap = a.pool_capacity;
+  if (int64_t(P.Hkv) * cap > INT32_MAX || int64_t(P.Hq) * 128 > INT32_MAX) return PSRL_ERR_SHAPE;
+  FwdMaps maps;
+  bool ok = make_map_bf16_2d(&maps.q, a.q, uint64_t(P.Hq) * 128, uint64_t(P.T_q), uint64_t(P.Hq) * 256, 128);
+  ok = ok && make_pool_maps(&maps.kv, a.k_pool, a.v_pool, P.Hkv, cap);
+  if (!ok) return PSRL_ERR_CUDA;
+  const DeviceHeader& H = P.hdr;
+  FwdParams p{};
+  p.blob = P.dev;
+  p.off_qt = H.off_qt; p.off_kvt = H.off_kvt; p.off_path_tiles = H.off_path_tiles;
+  p.off_path_nvalid = H.off_path_nvalid; p.off_page_slot = H.off_page_slot;
+  p.Hq = P.Hq; p.Hkv = P.Hkv; p.G = P.Hq / P.Hkv; p.T_q = P.T_q;
+  p.pairs_per_group = (p.G + NQ - 1) / NQ;
+  p.cap = cap;
+  p.scale_log2 = a.scale * kLog2e;
+  p.o = static_cast<__nv_bfloat16*>(a.o_out);
+  p.lse = a.lse_out;
+  p.status = a.status;
+  const size_t smem = size_t(NQ + KS + VS) * kTileBytes + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    if (e != cudaSuccess) { set_last_cuda_error(e); return PSRL_ERR_CUDA; }
+    attr_set = true;
+  }
+  const int64_t grid = int64_t(P.q_tiles.size()) * P.Hkv * p.pairs_per_group;
+  if (grid == 0) return PSRL_OK;
+  if (grid > INT32_MAX) return PSRL_ERR_SHAPE;
+  fwd_kernel<<<unsigned(grid), kThreads, smem, a.stream>>>(maps, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { set_last_cuda_error(e); return PSRL_ERR_CUDA; }
+  return PSRL_OK;
+}
+
+}  // namespace psrl

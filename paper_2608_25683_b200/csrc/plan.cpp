@@ -264,6 +264,7 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
           kt.n_pages = 1;
           kt.row_off = tok0 % bs;
           kt.rows_loaded = kTile;
+          kt.zero_rows = (bs > kTile && kt.row_off == 0 && t == nt - 1) ? bs - kTile : 0;
         } else {
           kt.first_page = P.seg_first_page[c] + tok0 / bs;
           kt.n_pages = (kt.n_valid + bs - 1) / bs;
@@ -374,6 +375,10 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
     H.off_kvi = append_array(B, P.kv_items);
     H.off_path_off = append_array(B, P.path_off);
     H.off_path_tiles = append_array(B, P.path_tiles);
+    P.path_nvalid.resize(P.path_tiles.size());
+    for (size_t i = 0; i < P.path_tiles.size(); ++i) P.path_nvalid[i] = P.kv_tiles[P.path_tiles[i]].n_valid;
+    H.off_path_nvalid = append_array(B, P.path_nvalid);
+    H.n_kvi = static_cast<int32_t>(P.kv_items.size());
     while (B.size() % 64) B.push_back(0);
     std::copy(reinterpret_cast<const int32_t*>(&H), reinterpret_cast<const int32_t*>(&H + 1), B.begin());
   } catch (const std::bad_alloc&) {

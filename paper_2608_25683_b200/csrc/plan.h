@@ -21,6 +21,9 @@ struct KvTile {
   int32_t seg;         // canonical segment
   int32_t tile_idx;    // index of the tile inside its segment
   int32_t rows_loaded; // rows a gather brings in: n_pages * min(bs, 128)
+  int32_t zero_rows;   // page slots after the tile's 128 rows that no tile covers (upper half of a 256-slot
+                       // page whose segment ends in the lower half): the backward writes zeros there
+  int32_t pad0, pad1, pad2;
 };
 
 // One query tile: up to 128 consecutive rows of one HAS_Q segment.
@@ -53,7 +56,9 @@ struct DeviceHeader {
   int32_t off_bt_off, off_bt_pages;
   int32_t off_qrow_seg;  // [T_q] segment of every query row
   int32_t off_kvt, off_qt, off_kvi, off_path_off, off_path_tiles;
-  int32_t reserved[8];
+  int32_t off_path_nvalid;  // valid keys of every entry of path_tiles
+  int32_t n_kvi;
+  int32_t reserved[6];
 };
 
 struct Plan {
@@ -72,7 +77,7 @@ struct Plan {
   std::vector<KvTile> kv_tiles;
   std::vector<QTile> q_tiles;    // longest first
   std::vector<KvItem> kv_items;  // longest first
-  std::vector<int32_t> seg_first_kvt, seg_n_kvt, seg_desc_q_begin, seg_desc_q_end, path_off, path_tiles, qrow_seg;
+  std::vector<int32_t> seg_first_kvt, seg_n_kvt, seg_desc_q_begin, seg_desc_q_end, path_off, path_tiles, path_nvalid, qrow_seg;
   // device blob
   std::vector<int32_t> blob;
   DeviceHeader hdr{};

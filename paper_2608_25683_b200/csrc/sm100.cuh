@@ -185,6 +185,12 @@ __device__ __forceinline__ uint32_t sw128_offset(int row, int col) {
   return uint32_t(row) * 128u + ((uint32_t(col >> 3) ^ (uint32_t(row) & 7u)) << 4) + (uint32_t(col) & 7u) * 2u;
 }
 
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
