@@ -1,0 +1,458 @@
+#!/usr/bin/env python
+"""Benchmark of tree-causal prefix-shared attention, forward + backward.
+
+Metric: fwd+bwd TFLOP/s over deduplicated FLOPs (14 * d * Hq * tree_pairs:
+forward 4d, backward 10d per attended (query, key) pair and query head; exact
+mask counts, no tile padding, no duplicated prefix work, no recompute).
+
+  python bench.py --gpus N --steps K --warmup W [--config c2] [--impl reference]
+
+One step = one pass of the whole hot path (forward, D pre-pass, dQ, dK/dV) over
+one synthetic batch.  N > 1 (torchrun): every rank runs an independent batch
+(prefix groups never span workers), no data-path collective, weak scaling.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "tree_attn_fwd_bwd_dedup_tflops"
+UNIT = "TFLOP/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel
+# (dkv_kernel), from the ncu captures summarised under profiles/ ; None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained"), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        # under load = the upper half of the samples (idle samples before/after the region are dropped)
+        sm_sorted = sorted(sm)
+        load = sm_sorted[len(sm_sorted) // 2:]
+        return {"sm_mhz": float(np.median(load)), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dedup_flops(d, Hq, pairs):
+    return 14.0 * d * Hq * float(pairs)
+
+
+# --------------------------------------------------------------------------- oracle legs
+def sub_workload(w, n_keep):
+    """The first `n_keep` samples of `w` (their root-to-end paths), as a workload."""
+    from paper_2608_25683_b200.workloads import Workload
+
+    n = len(w.parent)
+    has_child = [False] * n
+    for p in w.parent:
+        if p >= 0:
+            has_child[p] = True
+    flags = w.seg_flags or [1 | (0 if has_child[s] else 2) for s in range(n)]
+    ends = [s for s in range(n) if flags[s] & 2][:n_keep]
+    keep = set()
+    for e in ends:
+        s = e
+        while s != -1:
+            keep.add(s)
+            s = w.parent[s]
+    order = sorted(keep)
+    new = {s: i for i, s in enumerate(order)}
+    parent = [(-1 if w.parent[s] == -1 else new[w.parent[s]]) for s in order]
+    roots_all = [s for s in range(n) if w.parent[s] == -1]
+    gbs = [w.group_block_size[roots_all.index(s)] for s in order if w.parent[s] == -1]
+    fl = [flags[s] if s in ends or not (flags[s] & 2) else flags[s] & ~2 for s in order]
+    # an interior segment whose kept children all vanished cannot happen: ends are kept whole paths
+    return Workload(w.name + f"[first {len(ends)} samples]", parent, [w.seg_len[s] for s in order], gbs,
+                    w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, seg_flags=fl, seed=w.seed)
+
+
+def oracle_leg(w, n_keep, seed, steps=1, warmup=0):
+    """Times the fp64 oracle, as it stands, on KV head 0 of the first n_keep samples."""
+    import torch
+    from oracle import oracle_attn, oracle_plan
+    from paper_2608_25683_b200.workloads import make_inputs
+
+    sw = sub_workload(w, n_keep)
+    plan = oracle_plan(sw.parent, sw.seg_len, sw.group_block_size, sw.seg_flags, None)
+    q, k, v, d_o = make_inputs(plan["T_q"], plan["pool_slots"], plan["tok_slot"], sw.n_q_heads, sw.n_kv_heads,
+                               sw.head_dim, sw.dtype, seed, device="cpu")
+    f = lambda t: t.float().numpy()
+    q, k, v, d_o = f(q), f(k), f(v), f(d_o)
+    G = sw.n_q_heads // sw.n_kv_heads
+    flops = dedup_flops(sw.head_dim, G, plan["tree_pairs"])
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle_attn(plan, q, k, v, d_o, sw.softmax_scale, kv_heads=[0])
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    t = float(np.mean(times))
+    cores = len(os.sched_getaffinity(0))
+    return dict(value=flops / t / 1e12, unit=UNIT, cores=cores, kind="oracle",
+                sample=f"KV head 0 ({G} query heads) of the first {plan['n_samples']} samples of {w.name} "
+                       f"(seed {w.seed}): {plan['T']} tree tokens, {plan['flat_tokens']} unshared tokens, "
+                       f"{flops:.3e} dedup FLOP, {t:.2f} s per pass (numpy fp64, torch threads "
+                       f"{torch.get_num_threads()})"), t
+
+
+def run_reference(args):
+    from paper_2608_25683_b200.workloads import make_workload
+
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = make_workload(args.config, args.seed)
+    base, t = oracle_leg(w, args.ref_samples, args.seed + 1, steps=args.steps, warmup=args.warmup)
+    line = dict(metric=METRIC, value=base["value"], unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=t * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", impl="reference",
+                config=workload_config(w, None), cpu_baseline=base,
+                e2e=dict(value=base["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, view):
+    c = {"workload": f"{w.name}: " + {
+        "c1": "tiny fp32 tree, 64-token prefix + 4 branches of 32",
+        "c2": "step-wise RL group, 8 samples sharing a 4096-token prefix, suffixes U{256..1024}",
+        "c2s": "cached 4096-token prefix + 8 suffixes U{1..8} (HBM-bound case)",
+        "c3": "depth-3 branching-4 tree, 64 leaves",
+        "c4": "mixed batch of 32 prefix groups, per-group block size {16,64,256}, fragmented pool",
+        "c5": "long-context group, 32768-token prefix + 64 branches U{1024..4096}",
+    }.get(w.name, w.name),
+        "seed": w.seed, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+        "block_sizes": sorted(set(w.group_block_size)),
+        "l2": "per-step working set exceeds the 126 MB L2 (inputs larger than L2); no explicit flush"}
+    if view is not None:
+        c.update(tree_tokens=view["T"], unshared_tokens=view["flat_tokens"], tree_pairs=view["tree_pairs"],
+                 unshared_pairs=view["flat_pairs"], n_segments=view["n_seg"], n_samples=view["n_samples"],
+                 prefix_match_rate=round(1 - view["T"] / view["flat_tokens"], 4))
+    return c
+
+
+# --------------------------------------------------------------------------- GPU arm
+class Runner:
+    """Holds one workload's plan, device tensors and preallocated outputs."""
+
+    def __init__(self, lib, w, seed, device, view_from=None, data=None):
+        import torch
+
+        self.lib, self.w = lib, w
+        self.plan = lib.Plan(w.parent, w.seg_len, w.group_block_size, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype,
+                             w.seg_flags, w.free_extents).upload(device)
+        V = self.plan.view
+        if data is None:
+            from paper_2608_25683_b200.workloads import make_inputs
+            cap = V["pool_slots"]
+            if w.free_extents:
+                cap = max(cap, max(a + c for a, c in w.free_extents))
+            data = make_inputs(V["T_q"], cap, V["tok_slot"], w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, seed,
+                               device=device)
+        self.q, self.k, self.v, self.d_o = data
+        self.o = torch.empty_like(self.q)
+        self.lse = torch.empty((w.n_q_heads, V["T_q"]), dtype=torch.float32, device=device)
+        self.dq = torch.empty_like(self.q)
+        self.dk = torch.zeros_like(self.k)
+        self.dv = torch.zeros_like(self.v)
+        self.scale = w.softmax_scale
+
+    def fwd(self):
+        self.lib.psrl_tree_attn_fwd(self.plan, self.q, self.k, self.v, self.scale, o=self.o, lse=self.lse)
+
+    def bwd(self):
+        self.lib.psrl_tree_attn_bwd(self.plan, self.q, self.k, self.v, self.o, self.lse, self.d_o, self.scale,
+                                    d_q=self.dq, dk_pool=self.dk, dv_pool=self.dv)
+
+    def step(self):
+        self.fwd()
+        self.bwd()
+
+
+def time_region(fn, iters, warmup=0):
+    import torch
+
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def flat_runner(lib, r, device, head_slice=None):
+    """The same kernels on the unshared layout: every sample a root of its own
+    holding copies of its tokens; dO goes to the first copy of each token."""
+    import torch
+    from paper_2608_25683_b200.workloads import Workload
+
+    V = r.plan.view
+    w = r.w
+    parent, seg_len, gbs, tok_src, first = lib.flatten_forest(V)
+    Hq, Hkv = w.n_q_heads, w.n_kv_heads
+    G = Hq // Hkv
+    hs = slice(None) if head_slice is None else slice(head_slice * G, (head_slice + 1) * G)
+    ks = slice(None) if head_slice is None else slice(head_slice, head_slice + 1)
+    fw = Workload(w.name + "-flat", parent, seg_len, gbs, Hq if head_slice is None else G,
+                  Hkv if head_slice is None else 1, w.head_dim, w.dtype)
+    fplan = lib.Plan(fw.parent, fw.seg_len, fw.group_block_size, fw.n_q_heads, fw.n_kv_heads, fw.head_dim, fw.dtype)
+    FV = fplan.view
+    # token -> query row of the tree layout
+    qrow = np.full(V["T"], -1, dtype=np.int64)
+    for c in range(V["n_seg"]):
+        if V["seg_q_off"][c] >= 0:
+            qrow[V["seg_tok_off"][c]:V["seg_tok_off"][c] + V["seg_len"][c]] = np.arange(
+                V["seg_q_off"][c], V["seg_q_off"][c] + V["seg_len"][c])
+    assert (qrow[tok_src] >= 0).all(), "the unshared comparison needs queries on every segment"
+    src_rows = torch.as_tensor(qrow[tok_src], device=device)
+    src_slots = torch.as_tensor(V["tok_slot"][tok_src].astype(np.int64), device=device)
+    dst_slots = torch.as_tensor(FV["tok_slot"].astype(np.int64), device=device)
+    q = r.q[src_rows][:, hs].contiguous()
+    d_o = r.d_o[src_rows][:, hs].contiguous()
+    d_o[torch.as_tensor(~first, device=device)] = 0
+    k = torch.zeros((fw.n_kv_heads, FV["pool_slots"], w.head_dim), dtype=r.k.dtype, device=device)
+    v = torch.zeros_like(k)
+    k[:, dst_slots] = r.k[ks][:, src_slots]
+    v[:, dst_slots] = r.v[ks][:, src_slots]
+    return Runner(lib, fw, 0, device, data=(q, k, v, d_o))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c2")
+    ap.add_argument("--seed", type=int, default=2000)
+    ap.add_argument("--cpu-samples", type=int, default=4, help="samples in the oracle's timed sample")
+    ap.add_argument("--ref-samples", type=int, default=2, help="samples per step of --impl reference")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-unshared", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_25683_b200 import binding as lib, build
+    from paper_2608_25683_b200.workloads import make_workload
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    build.build()
+
+    # every rank gets an independent batch of the same shape (groups never span workers)
+    w = make_workload(args.config, args.seed + rank)
+    r = Runner(lib, w, args.seed + 1 + rank, device)
+    V = r.plan.view
+    flops = dedup_flops(w.head_dim, w.n_q_heads, V["tree_pairs"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        # the sampler also sees the warm-up so that short timed regions still get samples under load
+        t_w = time.perf_counter()
+        n_w = 0
+        while n_w < max(args.warmup, 3) or time.perf_counter() - t_w < 0.5:
+            r.step()
+            n_w += 1
+            if n_w % 8 == 0:
+                torch.cuda.synchronize()
+        assert lib.psrl_device_status(r.plan, "bwd") == 0
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            r.step()
+        e1.record()
+        barrier()
+    ms = e0.elapsed_time(e1) / args.steps
+    t = torch.tensor([ms, flops], dtype=torch.float64, device=device)
+    if world > 1:
+        tmax = t.clone()
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        tsum = t.clone()
+        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+        ms_max, flops_all = float(tmax[0]), float(tsum[1])
+    else:
+        ms_max, flops_all = ms, flops
+    value = flops_all / (ms_max * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    # ---- per-kernel times (each kernel alone, CUDA events on the launch stream) ----
+    it = max(5, min(args.steps, 20))
+    t_fwd = time_region(r.fwd, it, 2)
+    kern = {}
+    for name, mask in (("delta_kernel", 1), ("dq_kernel", 2), ("dkv_kernel", 4)):
+        lib.psrl_profile_bwd_phases(mask)
+        kern[name] = time_region(r.bwd, it, 2)
+    lib.psrl_profile_bwd_phases(7)
+    kern["fwd_kernel"] = t_fwd
+    d, Hq, pairs = w.head_dim, w.n_q_heads, float(V["tree_pairs"])
+    kflops = {"fwd_kernel": 4 * d * Hq * pairs, "dq_kernel": 2 * d * Hq * pairs, "dkv_kernel": 8 * d * Hq * pairs}
+    kernels = {}
+    for name, tms in kern.items():
+        kernels[name] = {"ms": round(tms, 4)}
+        if name in kflops:
+            kernels[name]["algorithmic_tflops"] = round(kflops[name] / (tms * 1e-3) / 1e12, 2)
+    es = 2 if w.dtype == "bf16" else 4
+    qbytes = V["T_q"] * Hq * d * es
+    kernels["delta_kernel"]["algorithmic_gbs"] = round((2 * qbytes + 4 * V["T_q"] * Hq) / (kern["delta_kernel"] * 1e-3) / 1e9, 1)
+    dom = max(("fwd_kernel", "dq_kernel", "dkv_kernel"), key=lambda n: kern[n])
+    achieved = kflops[dom] / (kern[dom] * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": round(achieved, 2), "peak": pk["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": round(achieved / pk["bf16_tflops"], 4),
+                "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+                "peak_source": f"{pk['source']} burst (kernel timed alone)", "kernels": kernels,
+                "whole_step_frac_of_burst": round(value / world / pk["bf16_tflops"], 4),
+                "whole_step_frac_of_sustained": round(value / world / pk["bf16_tflops_sustained"], 4)}
+    if w.dtype != "bf16":
+        roofline["bound"] = "alu"
+
+    # ---- end to end through the public call with host buffers ----
+    hq, hk, hv, hdo = (x.cpu().pin_memory() for x in (r.q, r.k, r.v, r.d_o))
+    ho, hl, hdq, hdk, hdv = (torch.empty_like(x, device="cpu").pin_memory() for x in (r.o, r.lse, r.dq, r.dk, r.dv))
+
+    def e2e_step():
+        r.q.copy_(hq, non_blocking=True); r.k.copy_(hk, non_blocking=True)
+        r.v.copy_(hv, non_blocking=True); r.d_o.copy_(hdo, non_blocking=True)
+        r.step()
+        ho.copy_(r.o, non_blocking=True); hl.copy_(r.lse, non_blocking=True); hdq.copy_(r.dq, non_blocking=True)
+        hdk.copy_(r.dk, non_blocking=True); hdv.copy_(r.dv, non_blocking=True)
+
+    e2e_ms = time_region(e2e_step, max(3, min(args.steps, 10)), 2)
+    nbytes = lambda *ts: int(sum(x.numel() * x.element_size() for x in ts))
+    e2e = {"value": round(flops / (e2e_ms * 1e-3) / 1e12 * world, 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
+           "h2d_bytes_per_step": nbytes(hq, hk, hv, hdo), "d2h_bytes_per_step": nbytes(ho, hl, hdq, hdk, hdv)}
+
+    # ---- the same kernels on the unshared (flattened) layout ----
+    unshared = None
+    if not args.no_unshared and world == 1:
+        try:
+            bytes_flat = V["flat_tokens"] * Hq * d * es * 4
+            slices = 1 if bytes_flat < 60e9 else w.n_kv_heads
+            t_flat = 0.0
+            for s in range(slices):
+                fr = flat_runner(lib, r, device, head_slice=None if slices == 1 else s)
+                t_flat += time_region(fr.step, max(3, min(args.steps, 10)), 2)
+                del fr
+                torch.cuda.empty_cache()
+            unshared = {"ms_per_step": round(t_flat, 3), "speedup_vs_unshared": round(t_flat / ms, 3),
+                        "flop_ratio_unshared_over_tree": round(V["flat_pairs"] / V["tree_pairs"], 3),
+                        "kv_head_slices": slices}
+        except Exception as ex:  # e.g. out of memory on the flattened tensors
+            unshared = {"error": str(ex)[:200]}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        cpu, _ = oracle_leg(w, args.cpu_samples, args.seed + 1)
+
+    line = dict(metric=METRIC, value=round(value, 3), unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=round(ms_max, 4), higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype=("bf16" if w.dtype == "bf16" else "f32"), data="synthetic",
+                config=workload_config(w, V), clocks=clocks.summary(), e2e=e2e, gpu_launches=4 * args.steps,
+                roofline=roofline, cpu_baseline=cpu, unshared=unshared,
+                frac_of_bf16_peak={"burst": round(value / world / pk["bf16_tflops"], 4),
+                                   "sustained": round(value / world / pk["bf16_tflops_sustained"], 4)})
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

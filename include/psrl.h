@@ -195,6 +195,16 @@ psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const v
  */
 psrl_status_t psrl_device_status(const void* workspace, void* stream);
 
+/*
+ * Profiling aid (no counterpart in the paper): restricts which kernels the
+ * NEXT psrl_tree_attn_bwd calls of this process launch, so that each backward
+ * kernel can be timed on its own with CUDA events.  Bit 0: D = rowsum(dO o O)
+ * pre-pass, bit 1: dQ kernel, bit 2: dK/dV kernel.  Default 7 (everything);
+ * with any other mask the skipped outputs are left untouched.  Returns the
+ * previous mask.  Not thread-safe; meant for benchmarks only.
+ */
+int psrl_profile_bwd_phases(int mask);
+
 /* Last CUDA error string seen by the library on this thread (HOST, static storage). */
 const char* psrl_last_cuda_error(void);
 

@@ -27,6 +27,7 @@ EXPORTS = [
     "psrl_plan_build", "psrl_plan_view", "psrl_plan_device_bytes", "psrl_plan_upload",
     "psrl_fwd_workspace_bytes", "psrl_bwd_workspace_bytes", "psrl_tree_attn_fwd", "psrl_tree_attn_bwd",
     "psrl_device_status", "psrl_last_cuda_error", "psrl_plan_destroy", "psrl_status_string",
+    "psrl_profile_bwd_phases",
 ]
 
 _I32P = C.POINTER(C.c_int32)
@@ -100,6 +101,8 @@ def lib() -> C.CDLL:
     L.psrl_tree_attn_bwd.restype = C.c_int
     L.psrl_device_status.argtypes = [C.c_void_p, C.c_void_p]
     L.psrl_device_status.restype = C.c_int
+    L.psrl_profile_bwd_phases.argtypes = [C.c_int]
+    L.psrl_profile_bwd_phases.restype = C.c_int
     L.psrl_last_cuda_error.restype = C.c_char_p
     L.psrl_plan_destroy.argtypes = [C.c_void_p]
     L.psrl_plan_destroy.restype = None
@@ -278,6 +281,12 @@ def psrl_tree_attn_bwd(plan: Plan, q, k_pool, v_pool, o, lse, d_o, softmax_scale
 def psrl_device_status(plan: Plan, kind: str = "fwd", stream=None, device="cuda") -> int:
     ws, _ = plan.workspace(kind, device)
     return int(lib().psrl_device_status(C.c_void_p(ws), _stream_ptr(stream)))
+
+
+def psrl_profile_bwd_phases(mask: int) -> int:
+    """Profiling aid: choose which backward kernels the next calls launch
+    (bit 0 delta pre-pass, bit 1 dQ, bit 2 dK/dV); returns the previous mask."""
+    return int(lib().psrl_profile_bwd_phases(int(mask)))
 
 
 def _check_dtype(plan: Plan, *tensors):

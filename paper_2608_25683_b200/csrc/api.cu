@@ -14,6 +14,7 @@ struct psrl_plan {
 namespace psrl {
 static thread_local cudaError_t g_last_cuda = cudaSuccess;
 void set_last_cuda_error(cudaError_t e) { g_last_cuda = e; }
+int g_bwd_phase_mask = 7;
 }  // namespace psrl
 
 namespace {
@@ -153,6 +154,12 @@ psrl_status_t psrl_device_status(const void* workspace, void* stream) {
   if (st == 0) return PSRL_OK;
   if (st == PSRL_ERR_TIMEOUT) return PSRL_ERR_TIMEOUT;
   return PSRL_ERR_INTERNAL;
+}
+
+int psrl_profile_bwd_phases(int mask) {
+  const int prev = psrl::g_bwd_phase_mask;
+  psrl::g_bwd_phase_mask = mask & 7;
+  return prev;
 }
 
 const char* psrl_last_cuda_error(void) { return cudaGetErrorString(psrl::g_last_cuda); }

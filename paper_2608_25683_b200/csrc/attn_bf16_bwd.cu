@@ -556,12 +556,14 @@ psrl_status_t bwd_bf16(const AttnArgs& a) {
     attr_set = true;
   }
 
-  if (P.T_q > 0) {
+  if (P.T_q > 0 && (g_bwd_phase_mask & 1)) {
     // ---- D = rowsum(dO o O) ----
     const int64_t units = int64_t(P.T_q) * P.Hq;
     delta_kernel<<<unsigned((units + 7) / 8), 256, 0, a.stream>>>(
         P.T_q, P.Hq, static_cast<const __nv_bfloat16*>(a.o), static_cast<const __nv_bfloat16*>(a.d_o), a.delta);
     if ((e = cudaGetLastError()) != cudaSuccess) return fail(e);
+  }
+  if (P.T_q > 0 && (g_bwd_phase_mask & 2)) {
     // ---- dQ ----
     dq::Params p{};
     p.blob = P.dev;
@@ -578,7 +580,7 @@ psrl_status_t bwd_bf16(const AttnArgs& a) {
       if ((e = cudaGetLastError()) != cudaSuccess) return fail(e);
     }
   }
-  {
+  if (g_bwd_phase_mask & 4) {
     // ---- dK, dV ----
     dkv::Maps km;
     if (P.T_q > 0) { km.q = qm.q; km.d_o = qm.d_o; }

@@ -32,4 +32,7 @@ psrl_status_t bwd_bf16(const AttnArgs& a);
 
 void set_last_cuda_error(cudaError_t e);
 
+// Which backward kernels to launch (profiling aid): bit 0 delta, bit 1 dQ, bit 2 dK/dV.
+extern int g_bwd_phase_mask;
+
 }  // namespace psrl
