@@ -33,7 +33,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel
 # (dkv_kernel), from the ncu captures summarised under profiles/ ; None = not captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"c2": 368589568 + 30693376}  # profiles/dkv_kernel_c2.md
 
 
 def peaks():
@@ -312,7 +312,7 @@ def main():
     import torch
     import torch.distributed as dist
 
-    from paper_2608_25683_b200 import binding as lib, build
+    from paper_2608_25683_b200 import binding as lib, build, dist_util
     from paper_2608_25683_b200.workloads import make_workload
 
     rank = int(os.environ.get("RANK", "0"))
@@ -327,8 +327,8 @@ def main():
     build.build()
 
     # every rank gets an independent batch of the same shape (groups never span workers)
-    w = make_workload(args.config, args.seed + rank)
-    r = Runner(lib, w, args.seed + 1 + rank, device)
+    w = make_workload(args.config, dist_util.rank_seed(args.seed, rank))
+    r = Runner(lib, w, dist_util.rank_seed(args.seed, rank) + 1, device)
     V = r.plan.view
     flops = dedup_flops(w.head_dim, w.n_q_heads, V["tree_pairs"])
 
@@ -355,15 +355,7 @@ def main():
         e1.record()
         barrier()
     ms = e0.elapsed_time(e1) / args.steps
-    t = torch.tensor([ms, flops], dtype=torch.float64, device=device)
-    if world > 1:
-        tmax = t.clone()
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = t.clone()
-        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        ms_max, flops_all = float(tmax[0]), float(tsum[1])
-    else:
-        ms_max, flops_all = ms, flops
+    ms_max, flops_all = dist_util.aggregate(ms, flops, device)  # max over ranks, sum of work
     value = flops_all / (ms_max * 1e-3) / 1e12
 
     if rank != 0:
