@@ -189,6 +189,45 @@ psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const v
                                  size_t workspace_bytes, void* stream);
 
 /*
+ * psrl_tree_attn_bwd_static - the backward pass for callers that cannot
+ * allocate device memory.  (The paper has no counterpart: this is a
+ * convenience of this library.)
+ *
+ * psrl_tree_attn_bwd needs a caller-provided device workspace.  Callers that
+ * must not call cudaMalloc - a latency-critical loop where an allocation would
+ * synchronise the device, a plug-in inside a process whose GPU memory belongs
+ * to another framework's pool, a process with a fixed memory budget - can use
+ * this variant instead: its workspace is a fixed array inside the library
+ * image (16 MiB + 256 bytes of device memory on every GPU that loads the
+ * library, held until the process exits).  The call itself performs no
+ * cudaMalloc / cudaFree and calls no allocating library routine.
+ *
+ * Same mathematics, same arguments and same results as psrl_tree_attn_bwd,
+ * except:
+ *   - no workspace arguments;
+ *   - limit: n_q_heads * T_q <= 4,194,304 (the array holds one float per query
+ *     row and head); larger plans return PSRL_ERR_WORKSPACE and must use
+ *     psrl_tree_attn_bwd;
+ *   - status_workspace (HOST pointer, may be NULL) receives the DEVICE address
+ *     of the array's status header; pass it to psrl_device_status to read the
+ *     launch's device status.
+ * Set-up: the first call on each device looks up the array's device address
+ * (with that device current) and caches it.  Make that first call outside any
+ * CUDA stream capture.
+ * Sharing: every call on a device uses the same array, which keeps the
+ * previous call's contents (the library clears what has to start at zero).
+ * Two calls that overlap on the GPU - different streams, or different host
+ * threads - race on it; serialise them, or use psrl_tree_attn_bwd with
+ * separate workspaces.
+ * Errors: INVALID_ARG, SHAPE, WORKSPACE (plan not uploaded, or over the
+ * limit), CUDA.  Asynchronous.
+ */
+psrl_status_t psrl_tree_attn_bwd_static(const psrl_plan_t* plan, const void* q, const void* k_pool,
+                                        const void* v_pool, int64_t pool_capacity, const void* o, const float* lse,
+                                        const void* d_o, void* d_q, void* dk_pool, void* dv_pool,
+                                        float softmax_scale, void** status_workspace, void* stream);
+
+/*
  * Synchronises `stream`, then reads the status word the last launch that used
  * `workspace` left: PSRL_OK, PSRL_ERR_TIMEOUT (a bounded wait gave up; outputs
  * are invalid) or PSRL_ERR_INTERNAL.  CUDA errors map to PSRL_ERR_CUDA.

@@ -27,7 +27,7 @@ EXPORTS = [
     "psrl_plan_build", "psrl_plan_view", "psrl_plan_device_bytes", "psrl_plan_upload",
     "psrl_fwd_workspace_bytes", "psrl_bwd_workspace_bytes", "psrl_tree_attn_fwd", "psrl_tree_attn_bwd",
     "psrl_device_status", "psrl_last_cuda_error", "psrl_plan_destroy", "psrl_status_string",
-    "psrl_profile_bwd_phases",
+    "psrl_profile_bwd_phases", "psrl_tree_attn_bwd_static",
 ]
 
 _I32P = C.POINTER(C.c_int32)
@@ -101,6 +101,10 @@ def lib() -> C.CDLL:
     L.psrl_tree_attn_bwd.restype = C.c_int
     L.psrl_device_status.argtypes = [C.c_void_p, C.c_void_p]
     L.psrl_device_status.restype = C.c_int
+    L.psrl_tree_attn_bwd_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
+                                            C.POINTER(C.c_void_p), C.c_void_p]
+    L.psrl_tree_attn_bwd_static.restype = C.c_int
     L.psrl_profile_bwd_phases.argtypes = [C.c_int]
     L.psrl_profile_bwd_phases.restype = C.c_int
     L.psrl_last_cuda_error.restype = C.c_char_p
@@ -281,6 +285,25 @@ def psrl_tree_attn_bwd(plan: Plan, q, k_pool, v_pool, o, lse, d_o, softmax_scale
 def psrl_device_status(plan: Plan, kind: str = "fwd", stream=None, device="cuda") -> int:
     ws, _ = plan.workspace(kind, device)
     return int(lib().psrl_device_status(C.c_void_p(ws), _stream_ptr(stream)))
+
+
+def psrl_tree_attn_bwd_static(plan: Plan, q, k_pool, v_pool, o, lse, d_o, softmax_scale: float, d_q, dk_pool,
+                              dv_pool, stream=None) -> int:
+    """Backward without any device allocation: for callers that may not touch
+    the CUDA allocator (see include/psrl.h).  Unlike psrl_tree_attn_bwd this
+    wrapper allocates nothing either, so every output tensor must be passed in.
+    The library's built-in scratch array serves as workspace; it is shared by
+    all calls on the device, so calls must not overlap on the GPU, and it caps
+    the problem at n_q_heads * T_q <= 4,194,304 (PSRL_ERR_WORKSPACE beyond).
+    Returns the device address of the status header (for psrl_device_status)."""
+    _check_dtype(plan, q, k_pool, v_pool, o, d_o, d_q, dk_pool, dv_pool)
+    ws = C.c_void_p()
+    st = lib().psrl_tree_attn_bwd_static(plan.handle, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(),
+                                         int(k_pool.shape[1]), o.data_ptr(), lse.data_ptr(), d_o.data_ptr(),
+                                         d_q.data_ptr(), dk_pool.data_ptr(), dv_pool.data_ptr(),
+                                         float(softmax_scale), C.byref(ws), _stream_ptr(stream))
+    _check(st, "psrl_tree_attn_bwd_static")
+    return int(ws.value or 0)
 
 
 def psrl_profile_bwd_phases(mask: int) -> int:
