@@ -23,7 +23,7 @@ bool aligned(const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>
 
 size_t ws_bytes(const psrl::Plan& P, bool bwd) {
   size_t n = psrl::kWsHeaderBytes;
-  if (bwd) n += (size_t(P.Hq) * size_t(P.T_q) * sizeof(float) + 255) / 256 * 256;
+  if (bwd) n += psrl::ws_delta_bytes(P) + psrl::ws_slab_bytes(P);
   return n;
 }
 
@@ -138,6 +138,7 @@ psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const v
   a.d_q = d_q; a.dk_pool = dk_pool; a.dv_pool = dv_pool;
   a.status = static_cast<int*>(workspace);
   a.delta = reinterpret_cast<float*>(static_cast<char*>(workspace) + psrl::kWsHeaderBytes);
+  a.slabs = reinterpret_cast<float*>(static_cast<char*>(workspace) + psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P));
   a.pool_capacity = pool_capacity; a.scale = softmax_scale; a.stream = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemsetAsync(workspace, 0, psrl::kWsHeaderBytes, a.stream);
   if (e != cudaSuccess) return cuda_status(e);

@@ -137,29 +137,31 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     if (lane == 0) {
       constexpr uint32_t idesc_kk = make_idesc(128, 128, 0, 0);  // S = Q K^T, dP = dO V^T
       constexpr uint32_t idesc_mn = make_idesc(128, 128, 0, 1);  // dQ = dS K, K is MN-major
+      // descriptor low words (address >> 4 | LBO field); per K step only a constant is added
+      const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), g_lo = desc_lo(smem_u32(sdO), 16);
+      const uint32_t k_lo = desc_lo(smem_u32(sK), 16), v_lo = desc_lo(smem_u32(sV), 16);
+      const uint32_t k_mn = desc_lo(smem_u32(sK), kHalfBytes);
       auto issue_s_dp = [&](int q, int ks) {
-        const uint32_t q0 = smem_u32(sQ + q * kTileBytes), k0 = smem_u32(sK + ks * kTileBytes);
-        const uint32_t g0 = smem_u32(sdO + q * kTileBytes), v0 = smem_u32(sV);
+        const uint32_t q0 = q_lo + q * (kTileBytes >> 4), k0 = k_lo + ks * (kTileBytes >> 4);
+        const uint32_t g0 = g_lo + q * (kTileBytes >> 4);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-          mma_ss(tmem + q * 256, make_desc(q0 + off, 16, 1024), make_desc(k0 + off, 16, 1024), idesc_kk, k > 0);
+          const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
+          mma_ss_lo(tmem + q * 256, q0 + off, k0 + off, idesc_kk, k > 0);
         }
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-          mma_ss(tmem + q * 256 + 128, make_desc(g0 + off, 16, 1024), make_desc(v0 + off, 16, 1024), idesc_kk, k > 0);
+          const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
+          mma_ss_lo(tmem + q * 256 + 128, g0 + off, v_lo + off, idesc_kk, k > 0);
         }
       };
       auto issue_dq = [&](int q, int ks) {
-        const uint32_t b0 = smem_u32(sK + ks * kTileBytes);
+        const uint32_t b0 = k_mn + ks * (kTileBytes >> 4);
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          mma_ts(tmem + q * 256, tmem + q * 256 + 128 + k * 8, make_desc(b0 + k * 2048, kHalfBytes, 1024), idesc_mn,
-                 k > 0);
+        for (int k = 0; k < 8; ++k) mma_ts_lo(tmem + q * 256, tmem + q * 256 + 128 + k * 8, b0 + k * 128, idesc_mn, k > 0);
       };
-      bool ok = mbar_wait(&bar.qdo_full, 0, abortp, p.status) && mbar_wait(&bar.k_full[0], 0, abortp, p.status) &&
-                mbar_wait(&bar.v_full, 0, abortp, p.status);
+      bool ok = mbar_wait_relaxed(&bar.qdo_full, 0, abortp, p.status) && mbar_wait_relaxed(&bar.k_full[0], 0, abortp, p.status) &&
+                mbar_wait_relaxed(&bar.v_full, 0, abortp, p.status);
       if (ok) {
         tc_fence_after();
         for (int q = 0; q < nq; ++q) { issue_s_dp(q, 0); mma_commit(&bar.sd_full[q]); }
@@ -168,7 +170,7 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       for (int j = 0; ok && j < n_tiles; ++j) {
         const int ks = j % KS;
         for (int q = 0; ok && q < nq; ++q) {
-          ok = mbar_wait(&bar.ds_ready[q], j & 1, abortp, p.status);
+          ok = mbar_wait_relaxed(&bar.ds_ready[q], j & 1, abortp, p.status);
           if (!ok) break;
           tc_fence_after();
           issue_dq(q, ks);
@@ -178,10 +180,10 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
         if (ok && j + 1 < n_tiles) {
           const int ks1 = (j + 1) % KS;
           for (int q = 0; ok && q < nq; ++q) {
-            ok = mbar_wait(&bar.x_free[q], j & 1, abortp, p.status);
+            ok = mbar_wait_relaxed(&bar.x_free[q], j & 1, abortp, p.status);
             if (ok && q == 0)
-              ok = mbar_wait(&bar.k_full[ks1], ((j + 1) / KS) & 1, abortp, p.status) &&
-                   mbar_wait(&bar.v_full, (j + 1) & 1, abortp, p.status);
+              ok = mbar_wait_relaxed(&bar.k_full[ks1], ((j + 1) / KS) & 1, abortp, p.status) &&
+                   mbar_wait_relaxed(&bar.v_full, (j + 1) & 1, abortp, p.status);
             if (!ok) break;
             tc_fence_after();
             issue_s_dp(q, ks1);
@@ -281,248 +283,6 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
 }
 }  // namespace dq
 
-// ============================================================================ dK / dV
-namespace dkv {
-constexpr int ST = 2;                         // (Q, dO) ring depth
-constexpr int kThreads = (8 + 2) * 32;        // 8 softmax warps + producer + MMA
-constexpr uint32_t TM_ST = 0, TM_DPT = 128, TM_DV = 256, TM_DK = 384;
-
-struct Maps {
-  CUtensorMap q, d_o;
-  PoolMaps kv;
-};
-struct Params {
-  const int32_t* blob;
-  int32_t off_kvi, off_kvt, off_page_slot;
-  int32_t Hq, Hkv, G, T_q;
-  int64_t cap;
-  float scale, scale_log2;
-  const float* lse;
-  const float* delta;
-  __nv_bfloat16 *dk, *dv;
-  int* status;
-};
-struct __align__(8) Barriers {
-  uint64_t kv_full, qd_full[ST], qd_empty[ST], st_full, pd_ready, acc_full, lse_ready;
-};
-
-__global__ void __launch_bounds__(kThreads, 1)
-dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sK = smem;
-  uint8_t* sV = sK + kTileBytes;
-  uint8_t* sQ = sV + kTileBytes;             // ST tiles
-  uint8_t* sdO = sQ + ST * kTileBytes;       // ST tiles
-  __shared__ Barriers bar;
-  __shared__ uint32_t s_tmem;
-  __shared__ int s_abort;
-  __shared__ float s_lse[2][128], s_dl[2][128];
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int item = blockIdx.x / p.Hkv, hk = blockIdx.x % p.Hkv;
-  const KvItem it = reinterpret_cast<const KvItem*>(p.blob + p.off_kvi)[item];
-  const KvTile kt = reinterpret_cast<const KvTile*>(p.blob + p.off_kvt)[it.kvt];
-  const int n_own = it.own_q_row0 >= 0 ? (it.own_q_end - it.own_q_row0 + 127) / 128 : 0;
-  const int n_desc = (it.desc_q_end - it.desc_q_begin + 127) / 128;
-  const int n_it = (n_own + n_desc) * p.G;
-
-  if (tid == 0) {
-    s_abort = 0;
-    mbar_init(&bar.kv_full, 1);
-    for (int i = 0; i < ST; ++i) { mbar_init(&bar.qd_full[i], 1); mbar_init(&bar.qd_empty[i], 1); }
-    mbar_init(&bar.st_full, 1); mbar_init(&bar.pd_ready, 256); mbar_init(&bar.acc_full, 1);
-    mbar_init(&bar.lse_ready, 256);
-    fence_mbar_init();
-  }
-  if (warp == 9) { tmem_alloc(&s_tmem, 512); tmem_relinquish(); }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = s_tmem;
-  volatile int* abortp = &s_abort;
-
-  // query tile t of this item: first row, valid rows, whether it is the diagonal tile
-  auto q_tile = [&](int t, int& row0, int& nvq, bool& diag) {
-    if (t < n_own) {
-      row0 = it.own_q_row0 + t * 128;
-      nvq = min(128, it.own_q_end - row0);
-      diag = (t == 0);
-    } else {
-      row0 = it.desc_q_begin + (t - n_own) * 128;
-      nvq = min(128, it.desc_q_end - row0);
-      diag = false;
-    }
-  };
-
-  if (warp == 8) {
-    // ======================= TMA producer =======================
-    if (lane == 0) {
-      const int32_t* page_slot = p.blob + p.off_page_slot;
-      const int64_t head_row0 = int64_t(hk) * p.cap;
-      // K and V complete on the same barrier: two expect_tx arrivals would over-count, so
-      // post the byte count once and issue both gathers against it
-      if (n_it > 0) {
-        mbar_expect_tx(&bar.kv_full, uint32_t(kt.rows_loaded) * 512u);
-        const int rows_per_box = kt.bs >= 128 ? 128 : kt.bs;
-        const int mi = map_index(kt.bs);
-        for (int i = 0; i < kt.n_pages; ++i) {
-          const int row = int(head_row0 + page_slot[kt.first_page + i] + kt.row_off);
-          uint8_t* dk_ = sK + i * rows_per_box * 128;
-          uint8_t* dv_ = sV + i * rows_per_box * 128;
-          tma_load_2d(dk_, &maps.kv.k[mi], &bar.kv_full, 0, row);
-          tma_load_2d(dk_ + kHalfBytes, &maps.kv.k[mi], &bar.kv_full, 64, row);
-          tma_load_2d(dv_, &maps.kv.v[mi], &bar.kv_full, 0, row);
-          tma_load_2d(dv_ + kHalfBytes, &maps.kv.v[mi], &bar.kv_full, 64, row);
-        }
-      }
-      for (int i = 0; i < n_it; ++i) {
-        const int st = i % ST, t = i / p.G, g = i % p.G;
-        int row0, nvq; bool diag;
-        q_tile(t, row0, nvq, diag);
-        if (i >= ST && !mbar_wait(&bar.qd_empty[st], ((i / ST) + 1) & 1, abortp, p.status)) break;
-        mbar_expect_tx(&bar.qd_full[st], 2 * kTileBytes);
-        load_row_tile(sQ + st * kTileBytes, &maps.q, &bar.qd_full[st], hk * p.G + g, row0);
-        load_row_tile(sdO + st * kTileBytes, &maps.d_o, &bar.qd_full[st], hk * p.G + g, row0);
-      }
-    }
-  } else if (warp == 9) {
-    // ======================= MMA issuer =======================
-    if (lane == 0) {
-      constexpr uint32_t idesc_kk = make_idesc(128, 128, 0, 0);  // S^T = K Q^T, dP^T = V dO^T
-      constexpr uint32_t idesc_mn = make_idesc(128, 128, 0, 1);  // dV += P^T dO, dK += dS^T Q
-      bool ok = n_it == 0 || mbar_wait(&bar.kv_full, 0, abortp, p.status);
-      const uint32_t k0 = smem_u32(sK), v0 = smem_u32(sV);
-      for (int i = 0; ok && i < n_it; ++i) {
-        const int st = i % ST;
-        ok = mbar_wait(&bar.qd_full[st], (i / ST) & 1, abortp, p.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t q0 = smem_u32(sQ + st * kTileBytes), g0 = smem_u32(sdO + st * kTileBytes);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-          mma_ss(tmem + TM_ST, make_desc(k0 + off, 16, 1024), make_desc(q0 + off, 16, 1024), idesc_kk, k > 0);
-        }
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-          mma_ss(tmem + TM_DPT, make_desc(v0 + off, 16, 1024), make_desc(g0 + off, 16, 1024), idesc_kk, k > 0);
-        }
-        mma_commit(&bar.st_full);
-        ok = mbar_wait(&bar.pd_ready, i & 1, abortp, p.status);
-        if (!ok) break;
-        tc_fence_after();
-        // P^T / dS^T sit as packed bf16 in the first 32 columns of each 64-column half
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t a_off = (k >> 2) * 64 + (k & 3) * 8;
-          mma_ts(tmem + TM_DV, tmem + TM_ST + a_off, make_desc(g0 + k * 2048, kHalfBytes, 1024), idesc_mn,
-                 (i > 0 || k > 0));
-        }
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t a_off = (k >> 2) * 64 + (k & 3) * 8;
-          mma_ts(tmem + TM_DK, tmem + TM_DPT + a_off, make_desc(q0 + k * 2048, kHalfBytes, 1024), idesc_mn,
-                 (i > 0 || k > 0));
-        }
-        mma_commit(&bar.qd_empty[st]);
-      }
-      if (ok) mma_commit(&bar.acc_full);
-    }
-  } else {
-    // ======================= softmax-backward warps (8) =======================
-    const int half = warp >> 2;                          // which 64 query columns
-    const int keyrow = (warp & 3) * 32 + lane;           // key inside the tile = TMEM lane
-    const uint32_t t_lane = tmem + (uint32_t((warp & 3) * 32) << 16);
-    bool ok = true;
-    for (int i = 0; i < n_it; ++i) {
-      const int t = i / p.G, g = i % p.G, h = hk * p.G + g, b = i & 1;
-      int row0, nvq; bool diag;
-      q_tile(t, row0, nvq, diag);
-      // stage LSE (log2 units) and D of the tile's query rows
-      if (tid < 128) s_lse[b][tid] = tid < nvq ? p.lse[int64_t(h) * p.T_q + row0 + tid] * kLog2e : CUDART_INF_F;
-      else s_dl[b][tid - 128] = (tid - 128) < nvq ? p.delta[int64_t(h) * p.T_q + row0 + tid - 128] : 0.f;
-      mbar_arrive(&bar.lse_ready);
-      ok = mbar_wait(&bar.lse_ready, i & 1, abortp, p.status) && mbar_wait(&bar.st_full, i & 1, abortp, p.status);
-      if (!ok) break;
-      tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        const int col0 = half * 64 + c * 32;
-        uint32_t s[32], dp[32], pk[16], dk[16];
-        tmem_ld32(t_lane + TM_ST + col0, s);
-        tmem_ld32(t_lane + TM_DPT + col0, dp);
-        tmem_wait_ld();
-#pragma unroll
-        for (int x = 0; x < 32; x += 2) {
-          const int q0i = col0 + x, q1i = col0 + x + 1;
-          const float p0 = ex2(fmaf(__uint_as_float(s[x]), p.scale_log2, -s_lse[b][q0i]));
-          const float p1 = ex2(fmaf(__uint_as_float(s[x + 1]), p.scale_log2, -s_lse[b][q1i]));
-          const bool v0 = q0i < nvq && (!diag || q0i >= keyrow);
-          const bool v1 = q1i < nvq && (!diag || q1i >= keyrow);
-          const float pp0 = v0 ? p0 : 0.f, pp1 = v1 ? p1 : 0.f;
-          const float d0 = v0 ? p0 * (__uint_as_float(dp[x]) - s_dl[b][q0i]) : 0.f;
-          const float d1 = v1 ? p1 * (__uint_as_float(dp[x + 1]) - s_dl[b][q1i]) : 0.f;
-          pk[x >> 1] = pack_bf16(pp0, pp1);
-          dk[x >> 1] = pack_bf16(d0, d1);
-        }
-        tmem_st16(t_lane + TM_ST + half * 64 + c * 16, pk);
-        tmem_st16(t_lane + TM_DPT + half * 64 + c * 16, dk);
-      }
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&bar.pd_ready);
-    }
-    // ---- epilogue: warps 0-3 write dV, warps 4-7 write dK (scaled); pads are zeros ----
-    if (ok && n_it > 0) ok = mbar_wait(&bar.acc_full, 0, abortp, p.status);
-    if (ok) {
-      tc_fence_after();
-      const int rows_per_box = kt.bs >= 128 ? 128 : kt.bs;
-      const bool in_pages = keyrow < kt.rows_loaded;
-      const bool valid = keyrow < kt.n_valid && n_it > 0;
-      int64_t slot = 0;
-      if (in_pages)
-        slot = (p.blob + p.off_page_slot)[kt.first_page + keyrow / rows_per_box] + kt.row_off + keyrow % rows_per_box;
-      __nv_bfloat16* out = (half == 0 ? p.dv : p.dk) + (int64_t(hk) * p.cap + slot) * 128;
-      const float mul = half == 0 ? 1.f : p.scale;
-      if (keyrow < kt.zero_rows) {  // slots of the page that lie beyond the segment's last tile
-        __nv_bfloat16* z = out + int64_t(128) * 128;
-#pragma unroll
-        for (int x = 0; x < 16; ++x) *reinterpret_cast<uint4*>(z + x * 8) = make_uint4(0, 0, 0, 0);
-      }
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        if (n_it > 0) {
-          tmem_ld32(t_lane + (half == 0 ? TM_DV : TM_DK) + c * 32, r);
-          tmem_wait_ld();
-        }
-        if (in_pages) {
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (valid) {
-              v.x = pack_bf16(__uint_as_float(r[8 * x + 0]) * mul, __uint_as_float(r[8 * x + 1]) * mul);
-              v.y = pack_bf16(__uint_as_float(r[8 * x + 2]) * mul, __uint_as_float(r[8 * x + 3]) * mul);
-              v.z = pack_bf16(__uint_as_float(r[8 * x + 4]) * mul, __uint_as_float(r[8 * x + 5]) * mul);
-              v.w = pack_bf16(__uint_as_float(r[8 * x + 6]) * mul, __uint_as_float(r[8 * x + 7]) * mul);
-            }
-            *reinterpret_cast<uint4*>(out + c * 32 + x * 8) = v;
-          }
-        }
-      }
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 9) {
-    tc_fence_after();
-    tmem_dealloc(tmem, 512);
-  }
-}
-}  // namespace dkv
-
 cudaError_t set_smem(const void* fn, size_t bytes) {
   return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes));
 }
@@ -549,10 +309,8 @@ psrl_status_t bwd_bf16(const AttnArgs& a) {
 
   static bool attr_set = false;
   const size_t smem_dq = size_t(2 * dq::NQ + dq::KS + 1) * kTileBytes + 1024;
-  const size_t smem_dkv = size_t(2 + 2 * dkv::ST) * kTileBytes + 1024;
   if (!attr_set) {
     if ((e = set_smem(reinterpret_cast<const void*>(dq::dq_kernel), smem_dq)) != cudaSuccess) return fail(e);
-    if ((e = set_smem(reinterpret_cast<const void*>(dkv::dkv_kernel), smem_dkv)) != cudaSuccess) return fail(e);
     attr_set = true;
   }
 
@@ -581,22 +339,9 @@ psrl_status_t bwd_bf16(const AttnArgs& a) {
     }
   }
   if (g_bwd_phase_mask & 4) {
-    // ---- dK, dV ----
-    dkv::Maps km;
-    if (P.T_q > 0) { km.q = qm.q; km.d_o = qm.d_o; }
-    km.kv = qm.kv;
-    dkv::Params p{};
-    p.blob = P.dev;
-    p.off_kvi = H.off_kvi; p.off_kvt = H.off_kvt; p.off_page_slot = H.off_page_slot;
-    p.Hq = P.Hq; p.Hkv = P.Hkv; p.G = G; p.T_q = P.T_q;
-    p.cap = cap; p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
-    p.lse = a.lse_in; p.delta = a.delta;
-    p.dk = static_cast<__nv_bfloat16*>(a.dk_pool); p.dv = static_cast<__nv_bfloat16*>(a.dv_pool);
-    p.status = a.status;
-    const int64_t grid = int64_t(P.kv_items.size()) * P.Hkv;
-    if (grid > INT32_MAX) return PSRL_ERR_SHAPE;
-    dkv::dkv_kernel<<<unsigned(grid), dkv::kThreads, smem_dkv, a.stream>>>(km, p);
-    if ((e = cudaGetLastError()) != cudaSuccess) return fail(e);
+    // ---- dK, dV (attn_bf16_dkv.cu) ----
+    const psrl_status_t st = dkv_bf16(a);
+    if (st != PSRL_OK) return st;
   }
   return PSRL_OK;
 }

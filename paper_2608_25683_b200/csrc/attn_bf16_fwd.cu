@@ -18,11 +18,13 @@
 //   S = Q K^T      tcgen05.mma, A and B from shared memory (K-major, 128B swizzle)
 //   O_tile = P V   tcgen05.mma, A = P from tensor memory, B = V (MN-major)
 // The MMA issuer alternates between the two heads, so the tensor cores work
-// on one head while the other head's warpgroup does its softmax.  Each softmax
-// thread keeps the running max / sum and the output row (128 fp32) in
-// registers; per-tile products are read back from tensor memory and folded in
-// with the rescale factor (online softmax; partial results merged by
-// log-sum-exp), so tensor memory never needs rescaling.
+// on one head while the other head's warpgroup does its softmax.  O accumulates
+// in tensor memory across the KV tiles (online softmax: per-tile partial
+// results are merged by log-sum-exp).  Each softmax thread owns one query row:
+// it reads the whole 128-wide score row in one round trip, keeps the running
+// sum and a reference maximum in registers, and moves that reference only when
+// the true maximum has grown by more than 2^8 - only then is the accumulator
+// row in tensor memory rescaled (rare after the first tiles).
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -126,22 +128,25 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);   // S = Q K^T, both K-major
       constexpr uint32_t idesc_o = make_idesc(128, 128, 0, 1);   // O = P V, V is MN-major
+      // descriptor low words (address >> 4 | LBO field); per K step only a constant is added
+      const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), k_lo = desc_lo(smem_u32(sK), 16);
+      const uint32_t v_mn = desc_lo(smem_u32(sV), kHalfBytes);
       auto issue_s = [&](int q, int ks) {
-        const uint32_t a0 = smem_u32(sQ + q * kTileBytes), b0 = smem_u32(sK + ks * kTileBytes);
+        const uint32_t a0 = q_lo + q * (kTileBytes >> 4), b0 = k_lo + ks * (kTileBytes >> 4);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-          mma_ss(tmem + q * 256, make_desc(a0 + off, 16, 1024), make_desc(b0 + off, 16, 1024), idesc_s, k > 0);
+          const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
+          mma_ss_lo(tmem + q * 256, a0 + off, b0 + off, idesc_s, k > 0);
         }
       };
-      auto issue_pv = [&](int q, int vs) {
-        const uint32_t b0 = smem_u32(sV + vs * kTileBytes);
+      auto issue_pv = [&](int q, int vs, bool first) {
+        const uint32_t b0 = v_mn + vs * (kTileBytes >> 4);
+        const uint32_t acc0 = first ? 0u : 1u;
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-          mma_ts(tmem + q * 256 + 128, tmem + q * 256 + k * 8, make_desc(b0 + k * 2048, kHalfBytes, 1024), idesc_o,
-                 k > 0);
+          mma_ts_lo(tmem + q * 256 + 128, tmem + q * 256 + k * 8, b0 + k * 128, idesc_o, k > 0 ? 1u : acc0);
       };
-      bool ok = mbar_wait(&bar.q_full, 0, abortp, p.status) && mbar_wait(&bar.k_full[0], 0, abortp, p.status);
+      bool ok = mbar_wait_relaxed(&bar.q_full, 0, abortp, p.status) && mbar_wait_relaxed(&bar.k_full[0], 0, abortp, p.status);
       if (ok) {
         tc_fence_after();
         for (int q = 0; q < nq; ++q) { issue_s(q, 0); mma_commit(&bar.s_full[q]); }
@@ -150,17 +155,16 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       for (int j = 0; ok && j < n_tiles; ++j) {
         const int vs = j % VS;
         for (int q = 0; ok && q < nq; ++q) {
-          ok = mbar_wait(&bar.p_ready[q], j & 1, abortp, p.status);
-          if (ok && j > 0) ok = mbar_wait(&bar.o_empty[q], (j - 1) & 1, abortp, p.status);
-          if (ok && q == 0) ok = mbar_wait(&bar.v_full[vs], (j / VS) & 1, abortp, p.status);
+          ok = mbar_wait_relaxed(&bar.p_ready[q], j & 1, abortp, p.status);
+          if (ok && q == 0) ok = mbar_wait_relaxed(&bar.v_full[vs], (j / VS) & 1, abortp, p.status);
           if (!ok) break;
           tc_fence_after();
-          issue_pv(q, vs);
+          issue_pv(q, vs, j == 0);
           mma_commit(&bar.o_full[q]);
           if (q == nq - 1) mma_commit(&bar.v_empty[vs]);
           if (j + 1 < n_tiles) {
             const int ks = (j + 1) % KS;
-            if (q == 0) ok = mbar_wait(&bar.k_full[ks], ((j + 1) / KS) & 1, abortp, p.status);
+            if (q == 0) ok = mbar_wait_relaxed(&bar.k_full[ks], ((j + 1) / KS) & 1, abortp, p.status);
             if (!ok) break;
             tc_fence_after();
             issue_s(q, ks);
@@ -175,10 +179,11 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
     const int q = warp >> 2;
     const int row = tid & 127;                                  // query row inside the tile
     const uint32_t t_lane = tmem + (uint32_t((warp & 3) * 32) << 16) + q * 256;
-    float acc[128];
-#pragma unroll
-    for (int i = 0; i < 128; ++i) acc[i] = 0.f;
-    float m_run = -CUDART_INF_F, l_run = 0.f, alpha_prev = 1.f;
+    // m_ref: the reference maximum (log2 units) the row's P values and running sum are
+    // expressed against.  It follows the true running maximum lazily: it only moves when
+    // the maximum has grown by more than 2^8, so the output accumulator in tensor memory
+    // is rescaled rarely (typically only on the first tiles) instead of once per tile.
+    float m_ref = -CUDART_INF_F, l_run = 0.f;
     bool ok = true;
     int nv_next = path_nvalid[0];
     for (int j = 0; j < n_tiles; ++j) {
@@ -187,54 +192,41 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       const bool diag = (j == n_tiles - 1);
       const int limit = diag ? min(row + 1, n_valid) : n_valid;  // keys [0, limit) are visible
       const bool need_mask = diag || n_valid < 128;
-      // ---- fold the previous tile's product into the running output ----
-      if (j > 0) {
-        ok = mbar_wait(&bar.o_full[q], (j - 1) & 1, abortp, p.status);
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tmem_ld32(t_lane + 128 + c * 32, r);
-          tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) acc[c * 32 + i] = fmaf(acc[c * 32 + i], alpha_prev, __uint_as_float(r[i]));
-        }
-        tc_fence_before();
-        mbar_arrive(&bar.o_empty[q]);
-      }
-      // ---- softmax of this tile ----
+      // ---- softmax of this tile: the whole score row in one round trip to tensor memory ----
       ok = mbar_wait(&bar.s_full[q], j & 1, abortp, p.status);
       if (!ok) break;
       tc_fence_after();
+      uint32_t s[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(t_lane + c * 32, s[c]);
+      tmem_wait_ld();
       float mx = -CUDART_INF_F;
+      if (need_mask) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(t_lane + c * 32, r);
-        tmem_wait_ld();
-        if (need_mask) {
+        for (int c = 0; c < 4; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (c * 32 + i < limit) ? __uint_as_float(r[i]) : -CUDART_INF_F);
-        } else {
+          for (int i = 0; i < 32; ++i)
+            mx = fmaxf(mx, (c * 32 + i < limit) ? __uint_as_float(s[c][i]) : -CUDART_INF_F);
+      } else {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
-        }
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < 32; i += 2)
+            mx = fmaxf(mx, fmaxf(__uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1])));
       }
-      const float m_new = fmaxf(m_run, mx * p.scale_log2);
-      // a row that sees no key yet keeps m = -inf; use 0 as the reference then so exp2 stays finite
-      const float m_ref = (m_new == -CUDART_INF_F) ? 0.f : m_new;
-      const float alpha = ex2(m_run - m_ref);
+      const float m_new = fmaxf(m_ref, mx * p.scale_log2);
+      const bool move = m_new > m_ref + 8.f;            // also true on the first tile (m_ref = -inf)
+      const bool any_move = __any_sync(0xffffffffu, move);
+      const float m_use = move ? m_new : m_ref;
+      const float alpha = ex2(m_ref - m_use);            // 1 if the reference stays, 0 on the first tile
       float sum = 0.f;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        uint32_t r[32], pk[16];
-        tmem_ld32(t_lane + c * 32, r);
-        tmem_wait_ld();
+        uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          float e0 = ex2(fmaf(__uint_as_float(r[i]), p.scale_log2, -m_ref));
-          float e1 = ex2(fmaf(__uint_as_float(r[i + 1]), p.scale_log2, -m_ref));
+          float e0 = ex2(fmaf(__uint_as_float(s[c][i]), p.scale_log2, -m_use));
+          float e1 = ex2(fmaf(__uint_as_float(s[c][i + 1]), p.scale_log2, -m_use));
           if (need_mask) {
             e0 = (c * 32 + i < limit) ? e0 : 0.f;
             e1 = (c * 32 + i + 1 < limit) ? e1 : 0.f;
@@ -245,8 +237,22 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
         tmem_st16(t_lane + c * 16, pk);
       }
       l_run = fmaf(l_run, alpha, sum);
-      m_run = m_new;
-      alpha_prev = alpha;
+      m_ref = m_use;
+      // ---- the reference moved: rescale the accumulated output in tensor memory ----
+      if (j > 0 && any_move) {
+        ok = mbar_wait(&bar.o_full[q], (j - 1) & 1, abortp, p.status);  // P V of the previous tile is complete
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_lane + 128 + c * 32, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+          tmem_st32(t_lane + 128 + c * 32, r);
+        }
+      }
       // V rows at or beyond n_valid (page pads, rows no page covers) must be zero before P V
       if (q == 0 && n_valid < 128) {
         ok = mbar_wait(&bar.v_full[j % VS], (j / VS) & 1, abortp, p.status);
@@ -273,18 +279,15 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
         tmem_wait_ld();
         uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float a0 = fmaf(acc[c * 32 + i], alpha_prev, __uint_as_float(r[i])) * inv;
-          const float a1 = fmaf(acc[c * 32 + i + 1], alpha_prev, __uint_as_float(r[i + 1])) * inv;
-          pk[i >> 1] = pack_bf16(a0, a1);
-        }
+        for (int i = 0; i < 32; i += 2)
+          pk[i >> 1] = pack_bf16(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
         if (store) {
 #pragma unroll
           for (int x = 0; x < 4; ++x)
             *reinterpret_cast<uint4*>(orow + c * 32 + x * 8) = make_uint4(pk[4 * x], pk[4 * x + 1], pk[4 * x + 2], pk[4 * x + 3]);
         }
       }
-      if (store) p.lse[int64_t(h) * p.T_q + qt.q_row0 + row] = (m_run + log2f(l_run)) * kLn2;
+      if (store) p.lse[int64_t(h) * p.T_q + qt.q_row0 + row] = (m_ref + log2f(l_run)) * kLn2;
     }
   }
   tc_fence_before();

@@ -9,6 +9,14 @@ namespace psrl {
 // Layout of the caller's workspace: [0, 256) control words (word 0 = device
 // status), then D = rowsum(dO o O) as fp32 [Hq, T_q] for the backward.
 constexpr size_t kWsHeaderBytes = 256;
+// After D: fp32 partial dV/dK slabs of split KV tiles, [slab][kv head][dV, dK][128][128].
+constexpr size_t kSlabBytes = size_t(2) * 128 * 128 * sizeof(float);
+inline size_t ws_delta_bytes(const Plan& P) {
+  return (size_t(P.Hq) * size_t(P.T_q) * sizeof(float) + 255) / 256 * 256;
+}
+inline size_t ws_slab_bytes(const Plan& P) {
+  return P.dtype == PSRL_BF16 ? size_t(P.n_slabs) * size_t(P.Hkv) * kSlabBytes : 0;
+}
 
 struct AttnArgs {
   const Plan* plan;
@@ -17,6 +25,7 @@ struct AttnArgs {
   void *o_out, *d_q, *dk_pool, *dv_pool;
   float* lse_out;
   float* delta;  // D, in the workspace
+  float* slabs;  // partial dV/dK slabs, in the workspace (bf16 path)
   int* status;   // device status word
   int64_t pool_capacity;
   float scale;
@@ -29,6 +38,7 @@ cudaError_t bwd_f32(const AttnArgs& a);
 // bf16 tensor-core path (tcgen05 / TMEM / TMA; head_dim 128)
 psrl_status_t fwd_bf16(const AttnArgs& a);
 psrl_status_t bwd_bf16(const AttnArgs& a);
+psrl_status_t dkv_bf16(const AttnArgs& a);  // the dK/dV part of bwd_bf16 (+ reduce of split tiles)
 
 void set_last_cuda_error(cudaError_t e);
 

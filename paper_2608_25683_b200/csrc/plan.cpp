@@ -318,8 +318,17 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
     }
     std::stable_sort(P.q_tiles.begin(), P.q_tiles.end(),
                      [](const QTile& a, const QTile& b) { return a.n_kv_tiles > b.n_kv_tiles; });
-    // dK/dV items, longest first
-    std::vector<int64_t> cost;
+    // dK/dV items.  Cost of a KV tile = number of 64-row query sub-tiles that attend to it
+    // (the exact pair count of Eq. 1's attention term, in tile units).  Tiles much heavier
+    // than an SM's fair share are split into parts so that the longest item cannot dominate
+    // the makespan; the list is then ordered longest first.
+    auto n_subs = [](const KvItem& it) {
+      int64_t n = (it.desc_q_end - it.desc_q_begin + kSubRows - 1) / kSubRows;
+      if (it.own_q_row0 >= 0) n += (it.own_q_end - it.own_q_row0 + kSubRows - 1) / kSubRows;
+      return static_cast<int32_t>(n);
+    };
+    std::vector<KvItem> whole;
+    int64_t total_sub = 0;
     for (size_t k = 0; k < P.kv_tiles.size(); ++k) {
       const KvTile& kt = P.kv_tiles[k];
       KvItem it{};
@@ -334,15 +343,36 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
       }
       it.desc_q_begin = P.seg_desc_q_begin[c];
       it.desc_q_end = P.seg_desc_q_end[c];
-      P.kv_items.push_back(it);
+      it.sub_begin = 0;
+      it.sub_end = n_subs(it);
+      it.slab = -1;
+      total_sub += it.sub_end;
+      whole.push_back(it);
     }
-    auto item_cost = [](const KvItem& it) {
-      int64_t cst = (it.desc_q_end - it.desc_q_begin + kTile - 1) / kTile;
-      if (it.own_q_row0 >= 0) cst += (it.own_q_end - it.own_q_row0 + kTile - 1) / kTile;
-      return cst;
-    };
-    std::stable_sort(P.kv_items.begin(), P.kv_items.end(),
-                     [&](const KvItem& a, const KvItem& b) { return item_cost(a) > item_cost(b); });
+    constexpr int64_t kSms = 148, kMinPart = 24;
+    const int64_t fair = (total_sub * P.Hkv + kSms - 1) / kSms;       // sub-tiles per SM if perfectly balanced
+    const int64_t part_max = std::max<int64_t>(kMinPart, fair / 2);
+    for (const KvItem& it : whole) {
+      const int32_t n = it.sub_end;
+      if (n <= part_max + part_max / 2) {
+        P.kv_items.push_back(it);
+        continue;
+      }
+      const int32_t parts = static_cast<int32_t>((n + part_max - 1) / part_max);
+      KvSplit sp{it.kvt, P.n_slabs, parts, 0};
+      for (int32_t a = 0; a < parts; ++a) {
+        KvItem part = it;
+        part.sub_begin = static_cast<int32_t>(int64_t(n) * a / parts);
+        part.sub_end = static_cast<int32_t>(int64_t(n) * (a + 1) / parts);
+        part.slab = P.n_slabs + a;
+        P.kv_items.push_back(part);
+      }
+      P.n_slabs += parts;
+      P.kv_splits.push_back(sp);
+    }
+    std::stable_sort(P.kv_items.begin(), P.kv_items.end(), [](const KvItem& a, const KvItem& b) {
+      return (a.sub_end - a.sub_begin) > (b.sub_end - b.sub_begin);
+    });
 
     // ---- device blob ----
     DeviceHeader& H = P.hdr;
@@ -379,6 +409,9 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
     for (size_t i = 0; i < P.path_tiles.size(); ++i) P.path_nvalid[i] = P.kv_tiles[P.path_tiles[i]].n_valid;
     H.off_path_nvalid = append_array(B, P.path_nvalid);
     H.n_kvi = static_cast<int32_t>(P.kv_items.size());
+    H.off_split = append_array(B, P.kv_splits);
+    H.n_split = static_cast<int32_t>(P.kv_splits.size());
+    H.n_slabs = P.n_slabs;
     while (B.size() % 64) B.push_back(0);
     std::copy(reinterpret_cast<const int32_t*>(&H), reinterpret_cast<const int32_t*>(&H + 1), B.begin());
   } catch (const std::bad_alloc&) {

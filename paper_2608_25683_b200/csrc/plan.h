@@ -37,13 +37,26 @@ struct QTile {
   int32_t pad0, pad1;
 };
 
-// One dK/dV work item: a KV tile and the query rows that attend to it.
+constexpr int kSubRows = 64;  // query rows per step of the dK/dV kernel
+
+// One dK/dV work item: a KV tile and (a contiguous part of) the query rows that
+// attend to it.  The rows are walked in sub-tiles of kSubRows: first the own
+// segment's rows from the tile's first key on, then the rows of all strict
+// descendants.  A heavy tile is split into several items over disjoint
+// sub-tile ranges; their fp32 partial sums go to slabs of the workspace and are
+// added in part order by the reduce kernel (fixed order, bitwise reproducible).
 struct KvItem {
   int32_t kvt;         // KV tile id
   int32_t own_q_row0;  // first own-segment query row (the tile's first key), -1 if the segment has no queries
   int32_t own_q_end;   // one past the segment's last query row
   int32_t desc_q_begin, desc_q_end;  // query rows of all strict descendants (contiguous), empty if none
-  int32_t pad0, pad1, pad2;
+  int32_t sub_begin, sub_end;        // this item's range of sub-tiles
+  int32_t slab;                      // partial-sum slab, or -1 if the item owns the tile and writes the output
+};
+
+// A KV tile whose work was split: its partial slabs [slab0, slab0 + n_parts).
+struct KvSplit {
+  int32_t kvt, slab0, n_parts, pad;
 };
 
 // Offsets (in int32 units from the start of the device blob) of each array.
@@ -58,7 +71,8 @@ struct DeviceHeader {
   int32_t off_kvt, off_qt, off_kvi, off_path_off, off_path_tiles;
   int32_t off_path_nvalid;  // valid keys of every entry of path_tiles
   int32_t n_kvi;
-  int32_t reserved[6];
+  int32_t n_split, off_split, n_slabs;
+  int32_t reserved[3];
 };
 
 struct Plan {
@@ -77,6 +91,8 @@ struct Plan {
   std::vector<KvTile> kv_tiles;
   std::vector<QTile> q_tiles;    // longest first
   std::vector<KvItem> kv_items;  // longest first
+  std::vector<KvSplit> kv_splits;
+  int32_t n_slabs = 0;
   std::vector<int32_t> seg_first_kvt, seg_n_kvt, seg_desc_q_begin, seg_desc_q_end, path_off, path_tiles, path_nvalid, qrow_seg;
   // device blob
   std::vector<int32_t> blob;
