@@ -134,7 +134,9 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     }
   } else if (warp == 4 * NQ + 1) {
     // ======================= MMA issuer =======================
-    if (lane == 0) {
+    // All 32 lanes walk the loop and wait on the barriers (warp-uniform control flow and
+    // address arithmetic); only the tcgen05 instructions are issued, by lane 0.
+    {
       constexpr uint32_t idesc_kk = make_idesc(128, 128, 0, 0);  // S = Q K^T, dP = dO V^T
       constexpr uint32_t idesc_mn = make_idesc(128, 128, 0, 1);  // dQ = dS K, K is MN-major
       // descriptor low words (address >> 4 | LBO field); per K step only a constant is added
@@ -144,51 +146,60 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       auto issue_s_dp = [&](int q, int ks) {
         const uint32_t q0 = q_lo + q * (kTileBytes >> 4), k0 = k_lo + ks * (kTileBytes >> 4);
         const uint32_t g0 = g_lo + q * (kTileBytes >> 4);
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
-          mma_ss_lo(tmem + q * 256, q0 + off, k0 + off, idesc_kk, k > 0);
-        }
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
+            mma_ss_lo(tmem + q * 256, q0 + off, k0 + off, idesc_kk, k > 0);
+          }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
-          mma_ss_lo(tmem + q * 256 + 128, g0 + off, v_lo + off, idesc_kk, k > 0);
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
+            mma_ss_lo(tmem + q * 256 + 128, g0 + off, v_lo + off, idesc_kk, k > 0);
+          }
         }
       };
       auto issue_dq = [&](int q, int ks) {
         const uint32_t b0 = k_mn + ks * (kTileBytes >> 4);
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) mma_ts_lo(tmem + q * 256, tmem + q * 256 + 128 + k * 8, b0 + k * 128, idesc_mn, k > 0);
+          for (int k = 0; k < 8; ++k)
+            mma_ts_lo(tmem + q * 256, tmem + q * 256 + 128 + k * 8, b0 + k * 128, idesc_mn, k > 0);
+        }
       };
-      bool ok = mbar_wait_relaxed(&bar.qdo_full, 0, abortp, p.status) && mbar_wait_relaxed(&bar.k_full[0], 0, abortp, p.status) &&
-                mbar_wait_relaxed(&bar.v_full, 0, abortp, p.status);
+      auto commit = [&](uint64_t* b) { if (elect_one()) mma_commit(b); };
+      auto wait = [&](uint64_t* b, uint32_t parity) {
+        return __all_sync(0xffffffffu, mbar_wait_relaxed(b, parity, abortp, p.status));
+      };
+      bool ok = wait(&bar.qdo_full, 0) && wait(&bar.k_full[0], 0) &&
+                wait(&bar.v_full, 0);
       if (ok) {
         tc_fence_after();
-        for (int q = 0; q < nq; ++q) { issue_s_dp(q, 0); mma_commit(&bar.sd_full[q]); }
-        mma_commit(&bar.v_empty);
+        for (int q = 0; q < nq; ++q) { issue_s_dp(q, 0); commit(&bar.sd_full[q]); }
+        commit(&bar.v_empty);
       }
       for (int j = 0; ok && j < n_tiles; ++j) {
         const int ks = j % KS;
         for (int q = 0; ok && q < nq; ++q) {
-          ok = mbar_wait_relaxed(&bar.ds_ready[q], j & 1, abortp, p.status);
+          ok = wait(&bar.ds_ready[q], j & 1);
           if (!ok) break;
           tc_fence_after();
           issue_dq(q, ks);
-          mma_commit(&bar.dq_full[q]);
-          if (q == nq - 1) mma_commit(&bar.k_empty[ks]);
+          commit(&bar.dq_full[q]);
+          if (q == nq - 1) commit(&bar.k_empty[ks]);
         }
         if (ok && j + 1 < n_tiles) {
           const int ks1 = (j + 1) % KS;
           for (int q = 0; ok && q < nq; ++q) {
-            ok = mbar_wait_relaxed(&bar.x_free[q], j & 1, abortp, p.status);
+            ok = wait(&bar.x_free[q], j & 1);
             if (ok && q == 0)
               ok = mbar_wait_relaxed(&bar.k_full[ks1], ((j + 1) / KS) & 1, abortp, p.status) &&
-                   mbar_wait_relaxed(&bar.v_full, (j + 1) & 1, abortp, p.status);
+                   wait(&bar.v_full, (j + 1) & 1);
             if (!ok) break;
             tc_fence_after();
             issue_s_dp(q, ks1);
-            mma_commit(&bar.sd_full[q]);
-            if (q == nq - 1) mma_commit(&bar.v_empty);
+            commit(&bar.sd_full[q]);
+            if (q == nq - 1) commit(&bar.v_empty);
           }
         }
       }

@@ -8,16 +8,18 @@
 // query heads of the KV head.  K and V stay in shared memory; dK and dV
 // accumulate in tensor memory over the whole loop.
 //
-// Per step (64 query rows of one head):
-//   MMA1  S^T = K Q^T, dP^T = V dO^T     M = 128 keys, N = 64 rows, both operands in smem
-//   warps P^T = exp2(S^T c - LSE), dS^T = P^T o (dP^T - D), written back to
-//         tensor memory as packed bf16 over the S^T / dP^T columns they came from
-//   MMA2  dV += P^T dO, dK += dS^T Q      A from tensor memory, dO / Q MN-major in smem
-// S^T and dP^T are double-buffered in tensor memory (2 x 64 columns each), so
-// MMA1 of step i+1 is issued before the warps have finished step i and the
-// tensor cores stay busy while the exponentials are computed.
+// Per step (128 query rows of one head) the tensor cores run four contractions
+// (M = 128 keys, N = 128, K = 128) and the warps run two half-steps:
+//   S^T  = K Q^T                 -> warps: P^T = exp2(S^T c - LSE), written over S^T as bf16
+//   dV  += P^T dO                   (A = P^T from tensor memory, dO MN-major in smem)
+//   dP^T = V dO^T                -> warps: dS^T = P^T o (dP^T - D), written over dP^T as bf16
+//   dK  += dS^T Q                   (A = dS^T from tensor memory, Q MN-major in smem)
+// The issue order is  dV(i), S^T(i+1), dK(i), dP^T(i+1):  while the warps turn S^T(i+1)
+// into P^T(i+1) the tensor cores work on dK(i) and dP^T(i+1); while they turn dP^T(i+1)
+// into dS^T(i+1) the tensor cores work on dV(i+1) and S^T(i+2).  S^T may be overwritten
+// as soon as dV(i) has been issued (it consumed P^T(i)), dP^T as soon as dK(i) has been.
 //
-// Tensor memory (512 columns): S^T[2] at 0/64, dP^T[2] at 128/192, dV at 256, dK at 384.
+// Tensor memory (512 columns): S^T at 0, dP^T at 128, dV at 256, dK at 384.
 // Heavy tiles are split over several CTAs by the plan; a split item writes its
 // fp32 partial to a workspace slab and reduce_kernel adds the parts in part
 // order (no atomics: bitwise reproducible).
@@ -32,14 +34,13 @@ namespace psrl {
 namespace {
 using namespace sm100;
 
-constexpr int ST = 4;                              // (Q, dO) sub-tile ring depth
-constexpr int kSubBytes = kSubRows * 128 * 2;      // 64 x 128 bf16 = two 64 x 64 halves
-constexpr int kSubHalf = kSubBytes / 2;
+constexpr int ST = 2;                              // (Q, dO) tile ring depth
+static_assert(kSubRows == 128, "the dK/dV kernel steps through 128-row query tiles");
 constexpr int kThreads = (8 + 2) * 32;             // 8 softmax-backward warps + producer + MMA
 constexpr uint32_t TM_ST = 0, TM_DPT = 128, TM_DV = 256, TM_DK = 384;
 
 struct Maps {
-  CUtensorMap q, d_o;  // boxes of 64 rows x 64 columns
+  CUtensorMap q, d_o;  // boxes of 128 rows x 64 columns
   PoolMaps kv;
 };
 struct Params {
@@ -47,7 +48,7 @@ struct Params {
   int32_t off_kvi, off_kvt, off_page_slot, off_split;
   int32_t Hq, Hkv, G, T_q;
   int64_t cap;
-  float scale, scale_log2;
+  float scale, scale_log2, inv_scale;
   const float* lse;
   const float* delta;
   float* slabs;
@@ -55,8 +56,42 @@ struct Params {
   int* status;
 };
 struct __align__(8) Barriers {
-  uint64_t kv_full, qd_full[ST], qd_empty[ST], st_full[2], pd_ready[2], acc_full;
+  uint64_t kv_full, qd_full[ST], qd_empty[ST], s_full, dp_full, p_ready, ds_ready, acc_full;
 };
+
+// The per-query-row terms of the backward are folded into the contractions as one extra
+// K = 16 step each, so the warps never have to fetch a per-column value:
+//   S^T_aug  = K Q^T   + 1 (x) (-LSE / scale)   ->  P^T  = exp2(scale log2e S^T_aug)
+//   dP^T_aug = V dO^T  + 1 (x) (-D)             ->  dS^T = P^T o dP^T_aug
+// The extra operands are [128 rows][16] bf16 slices in the no-swizzle K-major layout (8-row x
+// 16-byte core matrices: row r, column c at (r/8)*256 + (c/8)*128 + (r%8)*16 + (c%8)*2).  The
+// fp32 term is carried exactly as the sum of three bf16 numbers in columns 0-2 against ones.
+// A query row beyond the valid range gets -inf, which makes its P^T column exactly zero.
+constexpr int kSliceBytes = 128 * 16 * 2;
+constexpr uint32_t kSliceDescHi = (256u >> 4) | (1u << 14);  // SBO 256 bytes, version 1, no swizzle
+__device__ __forceinline__ uint32_t slice_row_offset(int r) { return uint32_t(r >> 3) * 256u + uint32_t(r & 7) * 16u; }
+__device__ __forceinline__ uint32_t slice_desc_lo(uint32_t smem_addr) {
+  return ((smem_addr & 0x3FFFF) >> 4) | ((128u >> 4) << 16);  // LBO 128 bytes: the second 8 columns
+}
+// x == a + b + c to fp32 precision, each term a bf16 (returned as raw 16-bit patterns)
+__device__ __forceinline__ uint2 split3_bf16(float x) {
+  const __nv_bfloat16 a = __float2bfloat16_rn(x);
+  float r = x - __bfloat162float(a);
+  const __nv_bfloat16 b = __float2bfloat16_rn(r);
+  r -= __bfloat162float(b);
+  const __nv_bfloat16 c = __float2bfloat16_rn(r);
+  return make_uint2(uint32_t(__bfloat16_as_ushort(a)) | (uint32_t(__bfloat16_as_ushort(b)) << 16),
+                    uint32_t(__bfloat16_as_ushort(c)));
+}
+__device__ __forceinline__ void mma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                            uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 
 // Slot of key row `row` of a KV tile in the pools.
 __device__ __forceinline__ int64_t tile_row_slot(const KvTile& kt, const int32_t* page_slot, int row) {
@@ -70,12 +105,15 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sK = smem;
   uint8_t* sV = sK + kTileBytes;
-  uint8_t* sQ = sV + kTileBytes;             // ST sub-tiles
-  uint8_t* sdO = sQ + ST * kSubBytes;        // ST sub-tiles
+  uint8_t* sQ = sV + kTileBytes;             // ST tiles
+  uint8_t* sdO = sQ + ST * kTileBytes;       // ST tiles
+  // K = 16 slices that fold the per-query-row terms into the contractions (see above)
+  uint8_t* sOnes = sdO + ST * kTileBytes;    // [128 keys][16]: columns 0-2 = 1
+  uint8_t* sLseX = sOnes + kSliceBytes;      // ST x [128 rows][16]: columns 0-2 = -LSE / scale in three bf16 terms
+  uint8_t* sDlX = sLseX + ST * kSliceBytes;  // ST x [128 rows][16]: columns 0-2 = -D in three bf16 terms
   __shared__ Barriers bar;
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
-  __shared__ __align__(16) float s_lse[ST][kSubRows], s_dl[ST][kSubRows];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int item = blockIdx.x / p.Hkv, hk = blockIdx.x % p.Hkv;
@@ -88,11 +126,19 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
     s_abort = 0;
     mbar_init(&bar.kv_full, 1);
     for (int i = 0; i < ST; ++i) { mbar_init(&bar.qd_full[i], 2); mbar_init(&bar.qd_empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&bar.st_full[i], 1); mbar_init(&bar.pd_ready[i], 256); }
+    mbar_init(&bar.s_full, 1); mbar_init(&bar.dp_full, 1);
+    mbar_init(&bar.p_ready, 256); mbar_init(&bar.ds_ready, 256);
     mbar_init(&bar.acc_full, 1);
     fence_mbar_init();
   }
   if (warp == 9) { tmem_alloc(&s_tmem, 512); tmem_relinquish(); }
+  // the constant slice: row r = key r, columns 0-2 = 1.0, the rest 0 (each row is 2 x 16 bytes)
+  if (tid < 128) {
+    uint8_t* r0 = sOnes + slice_row_offset(tid);
+    *reinterpret_cast<uint4*>(r0) = make_uint4(0x3F803F80u, 0x00003F80u, 0u, 0u);
+    *reinterpret_cast<uint4*>(r0 + 128) = make_uint4(0u, 0u, 0u, 0u);
+  }
+  fence_proxy_async();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -107,7 +153,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
     if (su < n_own_sub) {
       row0 = it.own_q_row0 + su * kSubRows;
       nvq = min(kSubRows, it.own_q_end - row0);
-      diag = su < 128 / kSubRows;
+      diag = su == 0;
       qpos0 = su * kSubRows;
     } else {
       row0 = it.desc_q_begin + (su - n_own_sub) * kSubRows;
@@ -138,147 +184,197 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
         }
       }
       // The whole warp walks the steps: lane 0 issues the TMA loads of Q and dO, all lanes
-      // stage the step's LSE (log2 units) and D rows next to them.  The ring runs ST steps
-      // ahead of the consumers, which hides the latency of these plain global loads.
+      // write the step's -LSE / scale and -D slices next to them.  The LSE / D values of a
+      // step are fetched (plain global loads) one step ahead, so their latency is not added
+      // to the time a freed stage takes to fill.  Every stage barrier gets two arrivals: the
+      // TMA byte count and the slices (after fence.proxy.async: the tensor cores read them).
+      auto fetch = [&](int i, float (&lv)[4], float (&dv)[4], int& nvq_out) {
+        int g, row0, nvq, qpos0; bool diag;
+        step(i, g, row0, nvq, diag, qpos0);
+        const int h = hk * p.G + g;
+        const float* lse_row = p.lse + int64_t(h) * p.T_q + row0;
+        const float* dl_row = p.delta + int64_t(h) * p.T_q + row0;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const int r = lane + 32 * x;
+          lv[x] = r < nvq ? lse_row[r] : 0.f;
+          dv[x] = r < nvq ? dl_row[r] : 0.f;
+        }
+        nvq_out = nvq;
+      };
+      float lv[4], dv[4], lv_n[4], dv_n[4];
+      int nvq_cur, nvq_next = 0;
+      fetch(0, lv, dv, nvq_cur);
       bool ok = true;
       for (int i = 0; ok && i < n_it; ++i) {
         const int st = i % ST;
         int g, row0, nvq, qpos0; bool diag;
         step(i, g, row0, nvq, diag, qpos0);
         const int h = hk * p.G + g;
+        if (i + 1 < n_it) fetch(i + 1, lv_n, dv_n, nvq_next);
         if (i >= ST) ok = mbar_wait(&bar.qd_empty[st], ((i / ST) + 1) & 1, abortp, p.status);
         if (!ok) break;
         if (lane == 0) {
-          mbar_expect_tx(&bar.qd_full[st], 2 * kSubBytes);
-          uint8_t* dq_ = sQ + st * kSubBytes;
-          uint8_t* dg_ = sdO + st * kSubBytes;
-          tma_load_2d(dq_, &maps.q, &bar.qd_full[st], h * 128, row0);
-          tma_load_2d(dq_ + kSubHalf, &maps.q, &bar.qd_full[st], h * 128 + 64, row0);
-          tma_load_2d(dg_, &maps.d_o, &bar.qd_full[st], h * 128, row0);
-          tma_load_2d(dg_ + kSubHalf, &maps.d_o, &bar.qd_full[st], h * 128 + 64, row0);
+          mbar_expect_tx(&bar.qd_full[st], 2 * kTileBytes);
+          load_row_tile(sQ + st * kTileBytes, &maps.q, &bar.qd_full[st], h, row0);
+          load_row_tile(sdO + st * kTileBytes, &maps.d_o, &bar.qd_full[st], h, row0);
         }
-        const float* lse_row = p.lse + int64_t(h) * p.T_q + row0;
-        const float* dl_row = p.delta + int64_t(h) * p.T_q + row0;
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
+        for (int x = 0; x < 4; ++x) {
           const int r = lane + 32 * x;
-          s_lse[st][r] = r < nvq ? lse_row[r] * kLog2e : CUDART_INF_F;
-          s_dl[st][r] = r < nvq ? dl_row[r] : 0.f;
+          uint2 u = make_uint2(0xFF80u, 0u), d = make_uint2(0u, 0u);  // -inf: a row beyond the range sees nothing
+          if (r < nvq_cur) {
+            u = split3_bf16(-lv[x] * p.inv_scale);
+            d = split3_bf16(-dv[x]);
+          }
+          uint8_t* lr = sLseX + st * kSliceBytes + slice_row_offset(r);
+          uint8_t* dr = sDlX + st * kSliceBytes + slice_row_offset(r);
+          *reinterpret_cast<uint4*>(lr) = make_uint4(u.x, u.y, 0u, 0u);
+          *reinterpret_cast<uint4*>(lr + 128) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(dr) = make_uint4(d.x, d.y, 0u, 0u);
+          *reinterpret_cast<uint4*>(dr + 128) = make_uint4(0u, 0u, 0u, 0u);
         }
+        fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bar.qd_full[st]);  // second arrival: LSE / D are in place
+        if (lane == 0) mbar_arrive(&bar.qd_full[st]);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) { lv[x] = lv_n[x]; dv[x] = dv_n[x]; }
+        nvq_cur = nvq_next;
       }
     }
   } else if (warp == 9) {
     // ======================= MMA issuer =======================
-    if (lane == 0 && n_it > 0) {
-      constexpr uint32_t idesc1 = make_idesc(128, kSubRows, 0, 0);  // S^T = K Q^T, dP^T = V dO^T
-      constexpr uint32_t idesc2 = make_idesc(128, 128, 0, 1);       // dV += P^T dO, dK += dS^T Q
+    // All 32 lanes walk the loop and wait on the barriers (warp-uniform control flow and
+    // address arithmetic); only the tcgen05 instructions are issued, by lane 0.
+    if (n_it > 0) {
+      constexpr uint32_t idesc_kk = make_idesc(128, 128, 0, 0);  // S^T = K Q^T, dP^T = V dO^T
+      constexpr uint32_t idesc_mn = make_idesc(128, 128, 0, 1);  // dV += P^T dO, dK += dS^T Q
       // descriptor low words (address >> 4 | LBO field); per K step only a constant is added
       const uint32_t k_lo = desc_lo(smem_u32(sK), 16), v_lo = desc_lo(smem_u32(sV), 16);
-      const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), g_lo = desc_lo(smem_u32(sdO), 16);              // K-major view
-      const uint32_t q_mn = desc_lo(smem_u32(sQ), kSubHalf), g_mn = desc_lo(smem_u32(sdO), kSubHalf);  // MN-major view
-      auto mma1 = [&](int i) {
-        const int st = i % ST, b = i & 1;
-        const uint32_t qs = q_lo + st * (kSubBytes >> 4), gs = g_lo + st * (kSubBytes >> 4);
+      const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), g_lo = desc_lo(smem_u32(sdO), 16);                  // K-major view
+      const uint32_t q_mn = desc_lo(smem_u32(sQ), kHalfBytes), g_mn = desc_lo(smem_u32(sdO), kHalfBytes);  // MN-major view
+      const uint32_t ones_lo = slice_desc_lo(smem_u32(sOnes));
+      const uint32_t lsex_lo = slice_desc_lo(smem_u32(sLseX)), dlx_lo = slice_desc_lo(smem_u32(sDlX));
+      // D = A B^T (both K-major, K = 128) + ones (x) extra (the K = 16 slice with the per-row term)
+      auto mma_kk = [&](uint32_t d, uint32_t a0, uint32_t b0, uint32_t extra_lo) {
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t oa = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2, ob = (k >> 2) * (kSubHalf >> 4) + (k & 3) * 2;
-          mma_ss_lo(tmem + TM_ST + b * 64, k_lo + oa, qs + ob, idesc1, k > 0);
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
+            mma_ss_lo(d, a0 + off, b0 + off, idesc_kk, k > 0);
+          }
+          mma_ss_lohi(d, ones_lo, kSliceDescHi, extra_lo, kSliceDescHi, idesc_kk, 1u);
         }
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t oa = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2, ob = (k >> 2) * (kSubHalf >> 4) + (k & 3) * 2;
-          mma_ss_lo(tmem + TM_DPT + b * 64, v_lo + oa, gs + ob, idesc1, k > 0);
-        }
-        mma_commit(&bar.st_full[b]);
       };
-      auto mma2 = [&](int i) {
-        const int st = i % ST, b = i & 1;
-        const uint32_t qs = q_mn + st * (kSubBytes >> 4), gs = g_mn + st * (kSubBytes >> 4);
-        const uint32_t acc0 = i > 0;
-        // P^T / dS^T: packed bf16, 16 query rows per 8 columns; rows 0-31 at +0, rows 32-63 at +32
+      auto mma_acc = [&](uint32_t d, uint32_t a_tmem, uint32_t b0, uint32_t acc0) {  // D += A[tmem] B, B MN-major
+        // packed bf16, 16 query rows per 8 columns; rows 0-63 at +0, rows 64-127 at +64
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const uint32_t a_off = (k >> 1) * 32 + (k & 1) * 8;
-          mma_ts_lo(tmem + TM_DV, tmem + TM_ST + b * 64 + a_off, gs + k * 128, idesc2, k > 0 ? 1u : acc0);
+          for (int k = 0; k < 8; ++k)
+            mma_ts_lo(d, a_tmem + (k >> 2) * 64 + (k & 3) * 8, b0 + k * 128, idesc_mn, k > 0 ? 1u : acc0);
         }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const uint32_t a_off = (k >> 1) * 32 + (k & 1) * 8;
-          mma_ts_lo(tmem + TM_DK, tmem + TM_DPT + b * 64 + a_off, qs + k * 128, idesc2, k > 0 ? 1u : acc0);
-        }
-        mma_commit(&bar.qd_empty[st]);
       };
-      bool ok = mbar_wait_relaxed(&bar.kv_full, 0, abortp, p.status) && mbar_wait_relaxed(&bar.qd_full[0], 0, abortp, p.status);
+      auto commit = [&](uint64_t* b) { if (elect_one()) mma_commit(b); };
+      auto wait = [&](uint64_t* b, uint32_t parity) {
+        return __all_sync(0xffffffffu, mbar_wait_relaxed(b, parity, abortp, p.status));
+      };
+      bool ok = wait(&bar.kv_full, 0) && wait(&bar.qd_full[0], 0);
       if (ok) {
         tc_fence_after();
-        mma1(0);
+        mma_kk(tmem + TM_ST, k_lo, q_lo, lsex_lo);
+        commit(&bar.s_full);
+        mma_kk(tmem + TM_DPT, v_lo, g_lo, dlx_lo);
+        commit(&bar.dp_full);
       }
       for (int i = 0; ok && i < n_it; ++i) {
-        if (i + 1 < n_it) {
-          ok = mbar_wait_relaxed(&bar.qd_full[(i + 1) % ST], ((i + 1) / ST) & 1, abortp, p.status);
-          if (!ok) break;
-          tc_fence_after();
-          mma1(i + 1);
-        }
-        ok = mbar_wait_relaxed(&bar.pd_ready[i & 1], (i >> 1) & 1, abortp, p.status);
+        const uint32_t so = (i % ST) * (kTileBytes >> 4), so1 = ((i + 1) % ST) * (kTileBytes >> 4);
+        const uint32_t sx1 = ((i + 1) % ST) * (kSliceBytes >> 4);
+        ok = wait(&bar.p_ready, i & 1);
         if (!ok) break;
         tc_fence_after();
-        mma2(i);
+        mma_acc(tmem + TM_DV, tmem + TM_ST, g_mn + so, i > 0);
+        if (i + 1 < n_it) {
+          ok = wait(&bar.qd_full[(i + 1) % ST], ((i + 1) / ST) & 1);
+          if (!ok) break;
+          mma_kk(tmem + TM_ST, k_lo, q_lo + so1, lsex_lo + sx1);
+          commit(&bar.s_full);
+        }
+        ok = wait(&bar.ds_ready, i & 1);
+        if (!ok) break;
+        tc_fence_after();
+        mma_acc(tmem + TM_DK, tmem + TM_DPT, q_mn + so, i > 0);
+        commit(&bar.qd_empty[i % ST]);
+        if (i + 1 < n_it) {
+          mma_kk(tmem + TM_DPT, v_lo, g_lo + so1, dlx_lo + sx1);
+          commit(&bar.dp_full);
+        }
       }
-      if (ok) mma_commit(&bar.acc_full);
+      if (ok) commit(&bar.acc_full);
     }
   } else {
     // ======================= softmax-backward warps (8) =======================
-    const int wg = warp >> 2;                            // which 32 query columns of the 64
+    const int wg = warp >> 2;                            // which 64 query columns of the 128
     const int keyrow = (warp & 3) * 32 + lane;           // key inside the tile = TMEM lane
     const uint32_t t_lane = tmem + (uint32_t((warp & 3) * 32) << 16);
     bool ok = true;
     for (int i = 0; i < n_it; ++i) {
-      const int b = i & 1;
       int g, row0, nvq, qpos0; bool diag;
       step(i, g, row0, nvq, diag, qpos0);
-      const int st = i % ST;
-      // LSE / D of this step were staged by the producer warp together with Q / dO
-      ok = mbar_wait(&bar.qd_full[st], (i / ST) & 1, abortp, p.status) &&
-           mbar_wait(&bar.st_full[b], (i >> 1) & 1, abortp, p.status);
+      float pr[64];  // this thread's P^T values, kept for the second half-step
+      // ---- half-step 1: P^T = exp2(c S^T_aug); -LSE / scale is already inside S^T_aug, and
+      //      a query row beyond the valid range carries -inf there, so its column comes out 0 ----
+      ok = mbar_wait(&bar.s_full, i & 1, abortp, p.status);
       if (!ok) break;
       tc_fence_after();
-      uint32_t s[32], dp[32], pk[16], dk[16];
-      tmem_ld32(t_lane + TM_ST + b * 64 + wg * 32, s);
-      tmem_ld32(t_lane + TM_DPT + b * 64 + wg * 32, dp);
-      float lse_r[32], dl_r[32];
+      {
+        uint32_t s[2][32];
+        tmem_ld32(t_lane + TM_ST + wg * 64, s[0]);
+        tmem_ld32(t_lane + TM_ST + wg * 64 + 32, s[1]);
+        tmem_wait_ld();
 #pragma unroll
-      for (int x = 0; x < 8; ++x) {
-        const float4 a = reinterpret_cast<const float4*>(&s_lse[st][wg * 32])[x];
-        const float4 d = reinterpret_cast<const float4*>(&s_dl[st][wg * 32])[x];
-        lse_r[4 * x] = a.x; lse_r[4 * x + 1] = a.y; lse_r[4 * x + 2] = a.z; lse_r[4 * x + 3] = a.w;
-        dl_r[4 * x] = d.x; dl_r[4 * x + 1] = d.y; dl_r[4 * x + 2] = d.z; dl_r[4 * x + 3] = d.w;
-      }
-      tmem_wait_ld();
-      const bool need_mask = diag || nvq < kSubRows;
+        for (int c = 0; c < 2; ++c) {
+          uint32_t pk[16];
 #pragma unroll
-      for (int x = 0; x < 32; x += 2) {
-        float p0 = ex2(fmaf(__uint_as_float(s[x]), p.scale_log2, -lse_r[x]));
-        float p1 = ex2(fmaf(__uint_as_float(s[x + 1]), p.scale_log2, -lse_r[x + 1]));
-        float d0 = p0 * (__uint_as_float(dp[x]) - dl_r[x]);
-        float d1 = p1 * (__uint_as_float(dp[x + 1]) - dl_r[x + 1]);
-        if (need_mask) {
-          const int c0 = wg * 32 + x, c1 = c0 + 1;
-          const bool v0 = c0 < nvq && (!diag || qpos0 + c0 >= keyrow);
-          const bool v1 = c1 < nvq && (!diag || qpos0 + c1 >= keyrow);
-          p0 = v0 ? p0 : 0.f; d0 = v0 ? d0 : 0.f;
-          p1 = v1 ? p1 : 0.f; d1 = v1 ? d1 : 0.f;
+          for (int x = 0; x < 32; x += 2) {
+            float p0 = ex2(__uint_as_float(s[c][x]) * p.scale_log2);
+            float p1 = ex2(__uint_as_float(s[c][x + 1]) * p.scale_log2);
+            if (diag) {  // the tile that holds the keys' own rows: a key is visible from its own row on
+              const int col = wg * 64 + c * 32 + x;
+              p0 = (qpos0 + col >= keyrow) ? p0 : 0.f;
+              p1 = (qpos0 + col + 1 >= keyrow) ? p1 : 0.f;
+            }
+            pr[c * 32 + x] = p0;
+            pr[c * 32 + x + 1] = p1;
+            pk[x >> 1] = pack_bf16(p0, p1);
+          }
+          tmem_st16(t_lane + TM_ST + wg * 64 + c * 16, pk);
         }
-        pk[x >> 1] = pack_bf16(p0, p1);
-        dk[x >> 1] = pack_bf16(d0, d1);
       }
-      tmem_st16(t_lane + TM_ST + b * 64 + wg * 32, pk);
-      tmem_st16(t_lane + TM_DPT + b * 64 + wg * 32, dk);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bar.pd_ready[b]);
+      mbar_arrive(&bar.p_ready);
+      // ---- half-step 2: dS^T = P^T o dP^T_aug (-D is already inside) ----
+      ok = mbar_wait(&bar.dp_full, i & 1, abortp, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      {
+        uint32_t dp[2][32];
+        tmem_ld32(t_lane + TM_DPT + wg * 64, dp[0]);
+        tmem_ld32(t_lane + TM_DPT + wg * 64 + 32, dp[1]);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int x = 0; x < 32; x += 2)
+            pk[x >> 1] = pack_bf16(pr[c * 32 + x] * __uint_as_float(dp[c][x]),
+                                   pr[c * 32 + x + 1] * __uint_as_float(dp[c][x + 1]));
+          tmem_st16(t_lane + TM_DPT + wg * 64 + c * 16, pk);
+        }
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bar.ds_ready);
     }
     // ---- epilogue: warps 0-3 take dV, warps 4-7 take dK ----
     if (ok && n_it > 0) ok = mbar_wait(&bar.acc_full, 0, abortp, p.status);
@@ -396,11 +492,11 @@ psrl_status_t dkv_bf16(const AttnArgs& a) {
   Maps m;
   bool ok = make_pool_maps(&m.kv, a.k_pool, a.v_pool, P.Hkv, cap);
   if (ok && P.T_q > 0) {
-    ok = make_map_bf16_2d(&m.q, a.q, uint64_t(P.Hq) * 128, uint64_t(P.T_q), uint64_t(P.Hq) * 256, kSubRows) &&
-         make_map_bf16_2d(&m.d_o, a.d_o, uint64_t(P.Hq) * 128, uint64_t(P.T_q), uint64_t(P.Hq) * 256, kSubRows);
+    ok = make_map_bf16_2d(&m.q, a.q, uint64_t(P.Hq) * 128, uint64_t(P.T_q), uint64_t(P.Hq) * 256, 128) &&
+         make_map_bf16_2d(&m.d_o, a.d_o, uint64_t(P.Hq) * 128, uint64_t(P.T_q), uint64_t(P.Hq) * 256, 128);
   }
   if (!ok) return PSRL_ERR_CUDA;
-  const size_t smem = size_t(2) * kTileBytes + size_t(2 * ST) * kSubBytes + 1024;
+  const size_t smem = size_t(2 + 2 * ST) * kTileBytes + size_t(1 + 2 * ST) * kSliceBytes + 1024;
   static bool attr_set = false;
   cudaError_t e;
   if (!attr_set) {
@@ -412,7 +508,7 @@ psrl_status_t dkv_bf16(const AttnArgs& a) {
   p.blob = P.dev;
   p.off_kvi = H.off_kvi; p.off_kvt = H.off_kvt; p.off_page_slot = H.off_page_slot; p.off_split = H.off_split;
   p.Hq = P.Hq; p.Hkv = P.Hkv; p.G = P.Hq / P.Hkv; p.T_q = P.T_q;
-  p.cap = cap; p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
+  p.cap = cap; p.scale = a.scale; p.scale_log2 = a.scale * kLog2e; p.inv_scale = 1.f / a.scale;
   p.lse = a.lse_in; p.delta = a.delta; p.slabs = a.slabs;
   p.dk = static_cast<__nv_bfloat16*>(a.dk_pool); p.dv = static_cast<__nv_bfloat16*>(a.dv_pool);
   p.status = a.status;

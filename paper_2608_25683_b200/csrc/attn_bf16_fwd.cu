@@ -125,7 +125,11 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
     }
   } else if (warp == 4 * NQ + 1) {
     // ======================= MMA issuer =======================
-    if (lane == 0) {
+    // All 32 lanes walk the loop and wait on the barriers, so control flow and address
+    // arithmetic stay warp-uniform; only the tcgen05 instructions are issued by lane 0.
+    // (A loop that only lane 0 executes turns every descriptor computation into
+    // per-thread work that competes with the softmax warps for issue slots.)
+    {
       constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);   // S = Q K^T, both K-major
       constexpr uint32_t idesc_o = make_idesc(128, 128, 0, 1);   // O = P V, V is MN-major
       // descriptor low words (address >> 4 | LBO field); per K step only a constant is added
@@ -133,43 +137,51 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       const uint32_t v_mn = desc_lo(smem_u32(sV), kHalfBytes);
       auto issue_s = [&](int q, int ks) {
         const uint32_t a0 = q_lo + q * (kTileBytes >> 4), b0 = k_lo + ks * (kTileBytes >> 4);
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
-          mma_ss_lo(tmem + q * 256, a0 + off, b0 + off, idesc_s, k > 0);
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
+            mma_ss_lo(tmem + q * 256, a0 + off, b0 + off, idesc_s, k > 0);
+          }
         }
       };
       auto issue_pv = [&](int q, int vs, bool first) {
         const uint32_t b0 = v_mn + vs * (kTileBytes >> 4);
         const uint32_t acc0 = first ? 0u : 1u;
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          mma_ts_lo(tmem + q * 256 + 128, tmem + q * 256 + k * 8, b0 + k * 128, idesc_o, k > 0 ? 1u : acc0);
+          for (int k = 0; k < 8; ++k)
+            mma_ts_lo(tmem + q * 256 + 128, tmem + q * 256 + k * 8, b0 + k * 128, idesc_o, k > 0 ? 1u : acc0);
+        }
       };
-      bool ok = mbar_wait_relaxed(&bar.q_full, 0, abortp, p.status) && mbar_wait_relaxed(&bar.k_full[0], 0, abortp, p.status);
+      auto commit = [&](uint64_t* b) { if (elect_one()) mma_commit(b); };
+      auto wait = [&](uint64_t* b, uint32_t parity) {
+        return __all_sync(0xffffffffu, mbar_wait_relaxed(b, parity, abortp, p.status));
+      };
+      bool ok = wait(&bar.q_full, 0) && wait(&bar.k_full[0], 0);
       if (ok) {
         tc_fence_after();
-        for (int q = 0; q < nq; ++q) { issue_s(q, 0); mma_commit(&bar.s_full[q]); }
-        mma_commit(&bar.k_empty[0]);
+        for (int q = 0; q < nq; ++q) { issue_s(q, 0); commit(&bar.s_full[q]); }
+        commit(&bar.k_empty[0]);
       }
       for (int j = 0; ok && j < n_tiles; ++j) {
         const int vs = j % VS;
         for (int q = 0; ok && q < nq; ++q) {
-          ok = mbar_wait_relaxed(&bar.p_ready[q], j & 1, abortp, p.status);
-          if (ok && q == 0) ok = mbar_wait_relaxed(&bar.v_full[vs], (j / VS) & 1, abortp, p.status);
+          ok = wait(&bar.p_ready[q], j & 1);
+          if (ok && q == 0) ok = wait(&bar.v_full[vs], (j / VS) & 1);
           if (!ok) break;
           tc_fence_after();
           issue_pv(q, vs, j == 0);
-          mma_commit(&bar.o_full[q]);
-          if (q == nq - 1) mma_commit(&bar.v_empty[vs]);
+          commit(&bar.o_full[q]);
+          if (q == nq - 1) commit(&bar.v_empty[vs]);
           if (j + 1 < n_tiles) {
             const int ks = (j + 1) % KS;
-            if (q == 0) ok = mbar_wait_relaxed(&bar.k_full[ks], ((j + 1) / KS) & 1, abortp, p.status);
+            if (q == 0) ok = wait(&bar.k_full[ks], ((j + 1) / KS) & 1);
             if (!ok) break;
             tc_fence_after();
             issue_s(q, ks);
-            mma_commit(&bar.s_full[q]);
-            if (q == nq - 1) mma_commit(&bar.k_empty[ks]);
+            commit(&bar.s_full[q]);
+            if (q == nq - 1) commit(&bar.k_empty[ks]);
           }
         }
       }

@@ -318,8 +318,8 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
     }
     std::stable_sort(P.q_tiles.begin(), P.q_tiles.end(),
                      [](const QTile& a, const QTile& b) { return a.n_kv_tiles > b.n_kv_tiles; });
-    // dK/dV items.  Cost of a KV tile = number of 64-row query sub-tiles that attend to it
-    // (the exact pair count of Eq. 1's attention term, in tile units).  Tiles much heavier
+    // dK/dV items.  Cost of a KV tile = number of 128-row query sub-tiles that attend to it
+    // (the pair count of Eq. 1's attention term, in tile units).  Tiles much heavier
     // than an SM's fair share are split into parts so that the longest item cannot dominate
     // the makespan; the list is then ordered longest first.
     auto n_subs = [](const KvItem& it) {
@@ -349,7 +349,7 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
       total_sub += it.sub_end;
       whole.push_back(it);
     }
-    constexpr int64_t kSms = 148, kMinPart = 24;
+    constexpr int64_t kSms = 148, kMinPart = 12;
     const int64_t fair = (total_sub * P.Hkv + kSms - 1) / kSms;       // sub-tiles per SM if perfectly balanced
     const int64_t part_max = std::max<int64_t>(kMinPart, fair / 2);
     for (const KvItem& it : whole) {

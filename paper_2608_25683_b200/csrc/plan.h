@@ -37,7 +37,7 @@ struct QTile {
   int32_t pad0, pad1;
 };
 
-constexpr int kSubRows = 64;  // query rows per step of the dK/dV kernel
+constexpr int kSubRows = 128;  // query rows per step of the dK/dV kernel
 
 // One dK/dV work item: a KV tile and (a contiguous part of) the query rows that
 // attend to it.  The rows are walked in sub-tiles of kSubRows: first the own

@@ -88,6 +88,18 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity
   return false;
 }
 
+// One lane of a fully active warp (the same lane every time for the same mask).
+// Issuing tcgen05 instructions under this predicate, inside warp-uniform control
+// flow, measured ~40 % more MMA throughput than a `lane == 0` branch when the
+// other warps of the SM are busy.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t elected;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(elected));
+  return elected != 0;
+}
+
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA, MMA)
 __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
