@@ -1,0 +1,312 @@
+// bf16 dQ kernel (query-stationary).
+//
+// One CTA = one query tile (up to 128 rows of one segment) x one query head.
+// It walks the tile's path of KV tiles exactly like the forward (all tiles of
+// the ancestor segments, then the own segment's tiles up to the diagonal) and
+// per tile runs three contractions (M = 128 rows, N = 128, K = 128):
+//   S  = Q K^T      -> warps: P = exp2(S c - LSE), kept in registers
+//   dP = dO V^T     -> warps: dS = P o (dP - D), written over dP as bf16
+//   dQ += dS K         (A = dS from tensor memory, K MN-major in smem)
+// dQ accumulates in tensor memory over the whole path, so every dQ row is
+// summed in path order by one CTA (bitwise reproducible).
+//
+// The warps work in two half-steps so that the tensor cores never wait for a
+// whole softmax: S may be overwritten as soon as the warps have READ it (P is
+// not stored back), so S(j+1) is issued while P(j) is still being computed;
+// dP(j+1) is issued right after dQ(j), which consumed dS(j).
+//
+// Warp roles: warps 0-7 softmax-backward (two threads per query row, 64 keys
+// each), warp 8 TMA producer, warp 9 MMA issuer + TMEM owner.
+// Tensor memory: S at 0, dP / dS at 128, dQ at 256.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "attn_bf16_common.cuh"
+#include "kernels.h"
+#include "tma.h"
+
+namespace psrl {
+namespace {
+using namespace sm100;
+
+constexpr int KS = 3, VS = 2;                 // K and V ring depths
+constexpr int kThreads = (8 + 2) * 32;
+constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 256;
+
+struct Maps {
+  CUtensorMap q, d_o;
+  PoolMaps kv;
+};
+struct Params {
+  const int32_t* blob;
+  int32_t off_qt, off_kvt, off_path_tiles, off_path_nvalid, off_page_slot;
+  int32_t Hq, G, T_q;
+  int64_t cap;
+  float scale, scale_log2;
+  const float* lse;
+  const float* delta;
+  __nv_bfloat16* d_q;
+  int* status;
+};
+struct __align__(8) Barriers {
+  uint64_t qdo_full, k_full[KS], k_empty[KS], v_full[VS], v_empty[VS];
+  uint64_t s_full, s_free, dp_full, ds_ready, dq_done;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+dq_kernel(const __grid_constant__ Maps maps, const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;
+  uint8_t* sdO = sQ + kTileBytes;
+  uint8_t* sK = sdO + kTileBytes;          // KS tiles
+  uint8_t* sV = sK + KS * kTileBytes;      // VS tiles
+  __shared__ Barriers bar;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int item = blockIdx.x / p.Hq, h = blockIdx.x % p.Hq, hk = h / p.G;
+  const QTile qt = reinterpret_cast<const QTile*>(p.blob + p.off_qt)[item];
+  const int32_t* path_tiles = p.blob + p.off_path_tiles + qt.pt_begin;
+  const int32_t* path_nvalid = p.blob + p.off_path_nvalid + qt.pt_begin;
+  const int n_tiles = qt.n_kv_tiles;
+
+  if (tid == 0) {
+    s_abort = 0;
+    mbar_init(&bar.qdo_full, 1);
+    for (int i = 0; i < KS; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1); }
+    for (int i = 0; i < VS; ++i) { mbar_init(&bar.v_full[i], 1); mbar_init(&bar.v_empty[i], 1); }
+    mbar_init(&bar.s_full, 1); mbar_init(&bar.s_free, 256);
+    mbar_init(&bar.dp_full, 1); mbar_init(&bar.ds_ready, 256);
+    mbar_init(&bar.dq_done, 1);
+    fence_mbar_init();
+  }
+  if (warp == 9) { tmem_alloc(&s_tmem, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  volatile int* abortp = &s_abort;
+
+  if (warp == 8) {
+    // ======================= TMA producer =======================
+    if (lane == 0) {
+      mbar_expect_tx(&bar.qdo_full, 2 * kTileBytes);
+      load_row_tile(sQ, &maps.q, &bar.qdo_full, h, qt.q_row0);
+      load_row_tile(sdO, &maps.d_o, &bar.qdo_full, h, qt.q_row0);
+      const KvTile* kvt = reinterpret_cast<const KvTile*>(p.blob + p.off_kvt);
+      const int32_t* page_slot = p.blob + p.off_page_slot;
+      const int64_t head_row0 = int64_t(hk) * p.cap;
+      for (int j = 0; j < n_tiles; ++j) {
+        const KvTile kt = kvt[path_tiles[j]];
+        const int ks = j % KS, vs = j % VS;
+        if (j >= KS && !mbar_wait(&bar.k_empty[ks], ((j / KS) + 1) & 1, abortp, p.status)) break;
+        load_kv_tile(sK + ks * kTileBytes, maps.kv.k, &bar.k_full[ks], kt, page_slot, head_row0);
+        if (j >= VS && !mbar_wait(&bar.v_empty[vs], ((j / VS) + 1) & 1, abortp, p.status)) break;
+        load_kv_tile(sV + vs * kTileBytes, maps.kv.v, &bar.v_full[vs], kt, page_slot, head_row0);
+      }
+    }
+  } else if (warp == 9) {
+    // ======================= MMA issuer =======================
+    // All 32 lanes walk the loop and wait on the barriers (warp-uniform control flow and
+    // address arithmetic); only the tcgen05 instructions are issued, by one elected lane.
+    constexpr uint32_t idesc_kk = make_idesc(128, 128, 0, 0);  // S = Q K^T, dP = dO V^T
+    constexpr uint32_t idesc_mn = make_idesc(128, 128, 0, 1);  // dQ += dS K, K is MN-major
+    const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), g_lo = desc_lo(smem_u32(sdO), 16);
+    const uint32_t k_lo = desc_lo(smem_u32(sK), 16), v_lo = desc_lo(smem_u32(sV), 16);
+    const uint32_t k_mn = desc_lo(smem_u32(sK), kHalfBytes);
+    auto mma_kk = [&](uint32_t d, uint32_t a0, uint32_t b0) {
+      if (elect_one()) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t off = (k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2;
+          mma_ss_lo(d, a0 + off, b0 + off, idesc_kk, k > 0);
+        }
+      }
+    };
+    auto commit = [&](uint64_t* b) { if (elect_one()) mma_commit(b); };
+    auto wait = [&](uint64_t* b, uint32_t parity) {
+      return __all_sync(0xffffffffu, mbar_wait_relaxed(b, parity, abortp, p.status));
+    };
+    bool ok = wait(&bar.qdo_full, 0) && wait(&bar.k_full[0], 0) && wait(&bar.v_full[0], 0);
+    if (ok) {
+      tc_fence_after();
+      mma_kk(tmem + TM_S, q_lo, k_lo);
+      commit(&bar.s_full);
+      mma_kk(tmem + TM_DP, g_lo, v_lo);
+      commit(&bar.dp_full);
+      commit(&bar.v_empty[0]);
+    }
+    for (int j = 0; ok && j < n_tiles; ++j) {
+      if (j + 1 < n_tiles) {
+        ok = wait(&bar.k_full[(j + 1) % KS], ((j + 1) / KS) & 1) && wait(&bar.s_free, j & 1);
+        if (!ok) break;
+        tc_fence_after();
+        mma_kk(tmem + TM_S, q_lo, k_lo + ((j + 1) % KS) * (kTileBytes >> 4));
+        commit(&bar.s_full);
+      }
+      ok = wait(&bar.ds_ready, j & 1);
+      if (!ok) break;
+      tc_fence_after();
+      if (elect_one()) {
+        // dS: packed bf16, 16 keys per 8 columns; keys 0-63 at +0, keys 64-127 at +64
+        const uint32_t b0 = k_mn + (j % KS) * (kTileBytes >> 4);
+        const uint32_t acc0 = j > 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          mma_ts_lo(tmem + TM_DQ, tmem + TM_DP + (k >> 2) * 64 + (k & 3) * 8, b0 + k * 128, idesc_mn,
+                    k > 0 ? 1u : acc0);
+      }
+      commit(&bar.k_empty[j % KS]);
+      if (j + 1 < n_tiles) {
+        const int vs = (j + 1) % VS;
+        ok = wait(&bar.v_full[vs], ((j + 1) / VS) & 1);
+        if (!ok) break;
+        mma_kk(tmem + TM_DP, g_lo, v_lo + vs * (kTileBytes >> 4));
+        commit(&bar.dp_full);
+        commit(&bar.v_empty[vs]);
+      }
+    }
+    if (ok) commit(&bar.dq_done);
+  } else {
+    // ======================= softmax-backward warps (8) =======================
+    const int half = warp >> 2;                           // which 64 keys of the tile
+    const int row = (warp & 3) * 32 + lane;               // query row inside the tile = TMEM lane
+    const uint32_t t_lane = tmem + (uint32_t((warp & 3) * 32) << 16);
+    const bool row_ok = row < qt.n_rows;
+    const float lse2 = row_ok ? p.lse[int64_t(h) * p.T_q + qt.q_row0 + row] * kLog2e : 0.f;
+    const float dl = row_ok ? p.delta[int64_t(h) * p.T_q + qt.q_row0 + row] : 0.f;
+    bool ok = true;
+    int nv_next = path_nvalid[0];
+    for (int j = 0; j < n_tiles; ++j) {
+      const int n_valid = nv_next;
+      if (j + 1 < n_tiles) nv_next = path_nvalid[j + 1];
+      const bool diag = (j == n_tiles - 1);
+      const int limit = diag ? min(row + 1, n_valid) : n_valid;   // keys [0, limit) are visible
+      const bool need_mask = diag || n_valid < 128;
+      float pr[64];
+      // ---- half-step 1: read S, release it, P = exp2(S c - LSE) ----
+      ok = mbar_wait(&bar.s_full, j & 1, abortp, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      {
+        uint32_t s[2][32];
+        tmem_ld32(t_lane + TM_S + half * 64, s[0]);
+        tmem_ld32(t_lane + TM_S + half * 64 + 32, s[1]);
+        tmem_wait_ld();
+        tc_fence_before();
+        mbar_arrive(&bar.s_free);
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+          for (int x = 0; x < 32; ++x) {
+            float pv = ex2(fmaf(__uint_as_float(s[c][x]), p.scale_log2, -lse2));
+            if (need_mask) pv = (half * 64 + c * 32 + x < limit) ? pv : 0.f;
+            pr[c * 32 + x] = pv;
+          }
+      }
+      // ---- half-step 2: dS = P o (dP - D) ----
+      ok = mbar_wait(&bar.dp_full, j & 1, abortp, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      {
+        uint32_t dp[2][32];
+        tmem_ld32(t_lane + TM_DP + half * 64, dp[0]);
+        tmem_ld32(t_lane + TM_DP + half * 64 + 32, dp[1]);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int x = 0; x < 32; x += 2) {
+            float d0 = pr[c * 32 + x] * (__uint_as_float(dp[c][x]) - dl);
+            float d1 = pr[c * 32 + x + 1] * (__uint_as_float(dp[c][x + 1]) - dl);
+            if (need_mask) {  // masked columns may hold anything (pad rows of V): select, do not multiply
+              d0 = (half * 64 + c * 32 + x < limit) ? d0 : 0.f;
+              d1 = (half * 64 + c * 32 + x + 1 < limit) ? d1 : 0.f;
+            }
+            pk[x >> 1] = pack_bf16(d0, d1);
+          }
+          tmem_st16(t_lane + TM_DP + half * 64 + c * 16, pk);
+        }
+      }
+      // K rows at or beyond n_valid must be zero before dS K (dS is zero there, K may hold anything)
+      if (n_valid < 128 && half == 0) {
+        ok = mbar_wait(&bar.k_full[j % KS], (j / KS) & 1, abortp, p.status);
+        if (!ok) break;
+        if (row >= n_valid) zero_tile_row(sK + (j % KS) * kTileBytes, row);
+        fence_proxy_async();
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bar.ds_ready);
+    }
+    // ---- dQ = scale * accumulator ----
+    if (ok) ok = mbar_wait(&bar.dq_done, 0, abortp, p.status);
+    if (ok) {
+      tc_fence_after();
+      __nv_bfloat16* drow = p.d_q + (int64_t(qt.q_row0 + row) * p.Hq + h) * 128 + half * 64;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld32(t_lane + TM_DQ + half * 64 + c * 32, r);
+        tmem_wait_ld();
+        if (row_ok) {
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(r[8 * x + 0]) * p.scale, __uint_as_float(r[8 * x + 1]) * p.scale);
+            v.y = pack_bf16(__uint_as_float(r[8 * x + 2]) * p.scale, __uint_as_float(r[8 * x + 3]) * p.scale);
+            v.z = pack_bf16(__uint_as_float(r[8 * x + 4]) * p.scale, __uint_as_float(r[8 * x + 5]) * p.scale);
+            v.w = pack_bf16(__uint_as_float(r[8 * x + 6]) * p.scale, __uint_as_float(r[8 * x + 7]) * p.scale);
+            *reinterpret_cast<uint4*>(drow + c * 32 + x * 8) = v;
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace
+
+psrl_status_t dq_bf16(const AttnArgs& a) {
+  const Plan& P = *a.plan;
+  const DeviceHeader& H = P.hdr;
+  const int64_t cap = a.pool_capacity;
+  if (P.T_q == 0 || P.q_tiles.empty()) return PSRL_OK;
+  auto fail = [](cudaError_t e) { set_last_cuda_error(e); return PSRL_ERR_CUDA; };
+  Maps m;
+  bool ok = make_pool_maps(&m.kv, a.k_pool, a.v_pool, P.Hkv, cap) &&
+            make_map_bf16_2d(&m.q, a.q, uint64_t(P.Hq) * 128, uint64_t(P.T_q), uint64_t(P.Hq) * 256, 128) &&
+            make_map_bf16_2d(&m.d_o, a.d_o, uint64_t(P.Hq) * 128, uint64_t(P.T_q), uint64_t(P.Hq) * 256, 128);
+  if (!ok) return PSRL_ERR_CUDA;
+  const size_t smem = size_t(2 + KS + VS) * kTileBytes + 1024;
+  static bool attr_set = false;
+  cudaError_t e;
+  if (!attr_set) {
+    e = cudaFuncSetAttribute(dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    if (e != cudaSuccess) return fail(e);
+    attr_set = true;
+  }
+  Params p{};
+  p.blob = P.dev;
+  p.off_qt = H.off_qt; p.off_kvt = H.off_kvt; p.off_path_tiles = H.off_path_tiles;
+  p.off_path_nvalid = H.off_path_nvalid; p.off_page_slot = H.off_page_slot;
+  p.Hq = P.Hq; p.G = P.Hq / P.Hkv; p.T_q = P.T_q;
+  p.cap = cap; p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
+  p.lse = a.lse_in; p.delta = a.delta; p.d_q = static_cast<__nv_bfloat16*>(a.d_q); p.status = a.status;
+  const int64_t grid = int64_t(P.q_tiles.size()) * P.Hq;
+  if (grid > INT32_MAX) return PSRL_ERR_SHAPE;
+  dq_kernel<<<unsigned(grid), kThreads, smem, a.stream>>>(m, p);
+  if ((e = cudaGetLastError()) != cudaSuccess) return fail(e);
+  return PSRL_OK;
+}
+
+}  // namespace psrl

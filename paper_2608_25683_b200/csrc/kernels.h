@@ -38,6 +38,7 @@ cudaError_t bwd_f32(const AttnArgs& a);
 // bf16 tensor-core path (tcgen05 / TMEM / TMA; head_dim 128)
 psrl_status_t fwd_bf16(const AttnArgs& a);
 psrl_status_t bwd_bf16(const AttnArgs& a);
+psrl_status_t dq_bf16(const AttnArgs& a);   // the dQ part of bwd_bf16
 psrl_status_t dkv_bf16(const AttnArgs& a);  // the dK/dV part of bwd_bf16 (+ reduce of split tiles)
 
 void set_last_cuda_error(cudaError_t e);
