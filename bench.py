@@ -33,7 +33,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel
 # (dkv_kernel), from the ncu captures summarised under profiles/ ; None = not captured.
-NCU_TRAFFIC_BYTES = {"c2": 368589568 + 30693376}  # profiles/dkv_kernel_c2.md
+NCU_TRAFFIC_BYTES = {"c2": 355098880 + 24278784}  # dram read + write of one dkv_kernel launch, profiles/dkv_kernel_c2.md
 
 
 def peaks():
@@ -375,7 +375,9 @@ def main():
     lib.psrl_profile_bwd_phases(7)
     kern["fwd_kernel"] = t_fwd
     d, Hq, pairs = w.head_dim, w.n_q_heads, float(V["tree_pairs"])
-    kflops = {"fwd_kernel": 4 * d * Hq * pairs, "dq_kernel": 2 * d * Hq * pairs, "dkv_kernel": 8 * d * Hq * pairs}
+    # contractions each kernel has to execute for its outputs (2*d flops per pair, head and contraction):
+    # forward S, PV; dQ kernel S, dP, dQ; dK/dV kernel S^T, dP^T, dV, dK.  The step metric counts 14*d (S and dP once).
+    kflops = {"fwd_kernel": 4 * d * Hq * pairs, "dq_kernel": 6 * d * Hq * pairs, "dkv_kernel": 8 * d * Hq * pairs}
     kernels = {}
     for name, tms in kern.items():
         kernels[name] = {"ms": round(tms, 4)}
@@ -436,7 +438,7 @@ def main():
     line = dict(metric=METRIC, value=round(value, 3), unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=round(ms_max, 4), higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype=("bf16" if w.dtype == "bf16" else "f32"), data="synthetic",
-                config=workload_config(w, V), clocks=clocks.summary(), e2e=e2e, gpu_launches=4 * args.steps,
+                config=workload_config(w, V), clocks=clocks.summary(), e2e=e2e, gpu_launches=(lib.psrl_launch_count(r.plan, False) + lib.psrl_launch_count(r.plan, True)) * args.steps,
                 roofline=roofline, cpu_baseline=cpu, unshared=unshared,
                 frac_of_bf16_peak={"burst": round(value / world / pk["bf16_tflops"], 4),
                                    "sustained": round(value / world / pk["bf16_tflops_sustained"], 4)})

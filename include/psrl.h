@@ -244,6 +244,15 @@ psrl_status_t psrl_device_status(const void* workspace, void* stream);
  */
 int psrl_profile_bwd_phases(int mask);
 
+/*
+ * Number of kernels one psrl_tree_attn_fwd (backward == 0) or
+ * psrl_tree_attn_bwd (backward != 0, all phases enabled) call launches for
+ * this plan (no counterpart in the paper; bookkeeping for benchmarks).
+ * Forward: 1.  Backward: D pre-pass + dQ + dK/dV, plus one fixed-order
+ * reduction when the bf16 schedule splits heavy KV tiles.  0 for a NULL plan.
+ */
+int psrl_launch_count(const psrl_plan_t* plan, int backward);
+
 /* Last CUDA error string seen by the library on this thread (HOST, static storage). */
 const char* psrl_last_cuda_error(void);
 

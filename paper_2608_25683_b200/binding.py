@@ -27,7 +27,7 @@ EXPORTS = [
     "psrl_plan_build", "psrl_plan_view", "psrl_plan_device_bytes", "psrl_plan_upload",
     "psrl_fwd_workspace_bytes", "psrl_bwd_workspace_bytes", "psrl_tree_attn_fwd", "psrl_tree_attn_bwd",
     "psrl_device_status", "psrl_last_cuda_error", "psrl_plan_destroy", "psrl_status_string",
-    "psrl_profile_bwd_phases", "psrl_tree_attn_bwd_static",
+    "psrl_profile_bwd_phases", "psrl_tree_attn_bwd_static", "psrl_launch_count",
 ]
 
 _I32P = C.POINTER(C.c_int32)
@@ -107,6 +107,8 @@ def lib() -> C.CDLL:
     L.psrl_tree_attn_bwd_static.restype = C.c_int
     L.psrl_profile_bwd_phases.argtypes = [C.c_int]
     L.psrl_profile_bwd_phases.restype = C.c_int
+    L.psrl_launch_count.argtypes = [C.c_void_p, C.c_int]
+    L.psrl_launch_count.restype = C.c_int
     L.psrl_last_cuda_error.restype = C.c_char_p
     L.psrl_plan_destroy.argtypes = [C.c_void_p]
     L.psrl_plan_destroy.restype = None
@@ -310,6 +312,11 @@ def psrl_profile_bwd_phases(mask: int) -> int:
     """Profiling aid: choose which backward kernels the next calls launch
     (bit 0 delta pre-pass, bit 1 dQ, bit 2 dK/dV); returns the previous mask."""
     return int(lib().psrl_profile_bwd_phases(int(mask)))
+
+
+def psrl_launch_count(plan: Plan, backward: bool) -> int:
+    """Kernels one forward (backward=False) or backward call launches for this plan."""
+    return int(lib().psrl_launch_count(plan._h, int(bool(backward))))
 
 
 def _check_dtype(plan: Plan, *tensors):

@@ -163,6 +163,12 @@ int psrl_profile_bwd_phases(int mask) {
   return prev;
 }
 
+int psrl_launch_count(const psrl_plan_t* plan, int backward) {
+  if (!plan || !plan->p) return 0;
+  if (!backward) return 1;
+  return 3 + ((plan->p->dtype == PSRL_BF16 && plan->p->n_slabs > 0) ? 1 : 0);
+}
+
 const char* psrl_last_cuda_error(void) { return cudaGetErrorString(psrl::g_last_cuda); }
 
 void psrl_plan_destroy(psrl_plan_t* plan) {
