@@ -123,6 +123,19 @@ psrl_status_t psrl_plan_build(const psrl_tree_desc_t* desc, psrl_plan_t** out_pl
 /* Fills *out with borrowed host pointers.  INVALID_ARG on NULL. */
 psrl_status_t psrl_plan_view(const psrl_plan_t* plan, psrl_plan_view_t* out);
 
+/*
+ * Borrowed HOST pointer to the device work schedule as psrl_plan_upload would
+ * copy it (int32 words; *n_words = psrl_plan_device_bytes / 4).  The layout is
+ * internal (a header of offsets, then the arrays: KV tiles, forward/dQ work
+ * items with their KV-tile lists, dK/dV work items and splits, merge lists)
+ * and not part of the bit-exact plan contract; it is exposed so that tests can
+ * check its invariants - every (query row, key) pair of the tree covered
+ * exactly once, every reduction a fixed total order (cf. the workload
+ * estimate of Eq. 1 that the schedule balances) - without a GPU.
+ * Valid until psrl_plan_destroy.  INVALID_ARG on NULL.
+ */
+psrl_status_t psrl_plan_schedule(const psrl_plan_t* plan, const int32_t** words, size_t* n_words);
+
 /* Bytes of DEVICE memory psrl_plan_upload needs (0 for a NULL plan). */
 size_t psrl_plan_device_bytes(const psrl_plan_t* plan);
 
@@ -248,8 +261,10 @@ int psrl_profile_bwd_phases(int mask);
  * Number of kernels one psrl_tree_attn_fwd (backward == 0) or
  * psrl_tree_attn_bwd (backward != 0, all phases enabled) call launches for
  * this plan (no counterpart in the paper; bookkeeping for benchmarks).
- * Forward: 1.  Backward: D pre-pass + dQ + dK/dV, plus one fixed-order
- * reduction when the bf16 schedule splits heavy KV tiles.  0 for a NULL plan.
+ * Forward: 1, plus a merge when rows are assembled from partial results
+ * (cascaded prefixes / split-KV).  Backward: D pre-pass + dQ + dK/dV, plus the
+ * dQ merge, plus one fixed-order reduction when the bf16 schedule splits
+ * heavy KV tiles.  0 for a NULL plan.
  */
 int psrl_launch_count(const psrl_plan_t* plan, int backward);
 

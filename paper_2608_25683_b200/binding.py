@@ -27,7 +27,7 @@ EXPORTS = [
     "psrl_plan_build", "psrl_plan_view", "psrl_plan_device_bytes", "psrl_plan_upload",
     "psrl_fwd_workspace_bytes", "psrl_bwd_workspace_bytes", "psrl_tree_attn_fwd", "psrl_tree_attn_bwd",
     "psrl_device_status", "psrl_last_cuda_error", "psrl_plan_destroy", "psrl_status_string",
-    "psrl_profile_bwd_phases", "psrl_tree_attn_bwd_static", "psrl_launch_count",
+    "psrl_profile_bwd_phases", "psrl_tree_attn_bwd_static", "psrl_launch_count", "psrl_plan_schedule",
 ]
 
 _I32P = C.POINTER(C.c_int32)
@@ -107,6 +107,8 @@ def lib() -> C.CDLL:
     L.psrl_tree_attn_bwd_static.restype = C.c_int
     L.psrl_profile_bwd_phases.argtypes = [C.c_int]
     L.psrl_profile_bwd_phases.restype = C.c_int
+    L.psrl_plan_schedule.argtypes = [C.c_void_p, C.POINTER(_I32P), C.POINTER(C.c_size_t)]
+    L.psrl_plan_schedule.restype = C.c_int
     L.psrl_launch_count.argtypes = [C.c_void_p, C.c_int]
     L.psrl_launch_count.restype = C.c_int
     L.psrl_last_cuda_error.restype = C.c_char_p
@@ -182,6 +184,12 @@ class Plan:
     @property
     def handle(self):
         return self._h
+
+    def schedule(self) -> np.ndarray:
+        """Copy of the device work schedule (int32 words) for host-side checks."""
+        words, n = _I32P(), C.c_size_t()
+        _check(lib().psrl_plan_schedule(self._h, C.byref(words), C.byref(n)), "psrl_plan_schedule")
+        return np.ctypeslib.as_array(words, shape=(n.value,)).copy()
 
     def device_bytes(self) -> int:
         return int(lib().psrl_plan_device_bytes(self._h))

@@ -23,7 +23,8 @@ bool aligned(const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>
 
 size_t ws_bytes(const psrl::Plan& P, bool bwd) {
   size_t n = psrl::kWsHeaderBytes;
-  if (bwd) n += psrl::ws_delta_bytes(P) + psrl::ws_slab_bytes(P);
+  if (bwd) n += psrl::ws_delta_bytes(P) + psrl::ws_slab_bytes(P) + psrl::ws_part_bytes(P);
+  else n += psrl::ws_part_bytes(P) + psrl::ws_part_lse_bytes(P);
   return n;
 }
 
@@ -76,6 +77,13 @@ psrl_status_t psrl_plan_view(const psrl_plan_t* plan, psrl_plan_view_t* v) {
   return PSRL_OK;
 }
 
+psrl_status_t psrl_plan_schedule(const psrl_plan_t* plan, const int32_t** words, size_t* n_words) {
+  if (!plan || !plan->p || !words || !n_words) return PSRL_ERR_INVALID_ARG;
+  *words = plan->p->blob.data();
+  *n_words = plan->p->blob.size();
+  return PSRL_OK;
+}
+
 size_t psrl_plan_device_bytes(const psrl_plan_t* plan) {
   if (!plan || !plan->p) return 0;
   return plan->p->blob.size() * sizeof(int32_t);
@@ -113,6 +121,8 @@ psrl_status_t psrl_tree_attn_fwd(const psrl_plan_t* plan, const void* q, const v
   psrl::AttnArgs a{};
   a.plan = &P; a.q = q; a.k_pool = k_pool; a.v_pool = v_pool; a.o_out = o; a.lse_out = lse;
   a.status = static_cast<int*>(workspace);
+  a.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + psrl::kWsHeaderBytes);
+  a.part_lse = reinterpret_cast<float*>(static_cast<char*>(workspace) + psrl::kWsHeaderBytes + psrl::ws_part_bytes(P));
   a.pool_capacity = pool_capacity; a.scale = softmax_scale; a.stream = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemsetAsync(workspace, 0, psrl::kWsHeaderBytes, a.stream);
   if (e != cudaSuccess) return cuda_status(e);
@@ -139,6 +149,8 @@ psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const v
   a.status = static_cast<int*>(workspace);
   a.delta = reinterpret_cast<float*>(static_cast<char*>(workspace) + psrl::kWsHeaderBytes);
   a.slabs = reinterpret_cast<float*>(static_cast<char*>(workspace) + psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P));
+  a.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P) +
+                                    psrl::ws_slab_bytes(P));
   a.pool_capacity = pool_capacity; a.scale = softmax_scale; a.stream = static_cast<cudaStream_t>(stream);
   cudaError_t e = cudaMemsetAsync(workspace, 0, psrl::kWsHeaderBytes, a.stream);
   if (e != cudaSuccess) return cuda_status(e);
@@ -165,8 +177,10 @@ int psrl_profile_bwd_phases(int mask) {
 
 int psrl_launch_count(const psrl_plan_t* plan, int backward) {
   if (!plan || !plan->p) return 0;
-  if (!backward) return 1;
-  return 3 + ((plan->p->dtype == PSRL_BF16 && plan->p->n_slabs > 0) ? 1 : 0);
+  const psrl::Plan& P = *plan->p;
+  const int merge = (P.dtype == PSRL_BF16 && !P.merge_row.empty()) ? 1 : 0;
+  if (!backward) return 1 + merge;
+  return 3 + ((P.dtype == PSRL_BF16 && P.n_slabs > 0) ? 1 : 0) + merge;
 }
 
 const char* psrl_last_cuda_error(void) { return cudaGetErrorString(psrl::g_last_cuda); }

@@ -46,6 +46,7 @@ struct Params {
   const float* lse;
   const float* delta;
   __nv_bfloat16* d_q;
+  float* part;  // unscaled fp32 dQ rows [n_part_rows][Hq][128] of items that do not own their rows
   int* status;
 };
 struct __align__(8) Barriers {
@@ -182,7 +183,7 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     for (int j = 0; j < n_tiles; ++j) {
       const int n_valid = nv_next;
       if (j + 1 < n_tiles) nv_next = path_nvalid[j + 1];
-      const bool diag = (j == n_tiles - 1);
+      const bool diag = qt.causal && (j == n_tiles - 1);
       const int limit = diag ? min(row + 1, n_valid) : n_valid;   // keys [0, limit) are visible
       const bool need_mask = diag || n_valid < 128;
       float pr[64];
@@ -252,7 +253,15 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
         uint32_t r[32];
         tmem_ld32(t_lane + TM_DQ + half * 64 + c * 32, r);
         tmem_wait_ld();
-        if (row_ok) {
+        if (row_ok && qt.part_row0 >= 0) {
+          // the row has other contributors: unscaled fp32 partial, summed by the merge kernel
+          float* prow = p.part + (int64_t(qt.part_row0 + row) * p.Hq + h) * 128 + half * 64 + c * 32;
+#pragma unroll
+          for (int x = 0; x < 8; ++x)
+            *reinterpret_cast<float4*>(prow + x * 4) =
+                make_float4(__uint_as_float(r[4 * x]), __uint_as_float(r[4 * x + 1]), __uint_as_float(r[4 * x + 2]),
+                            __uint_as_float(r[4 * x + 3]));
+        } else if (row_ok) {
 #pragma unroll
           for (int x = 0; x < 4; ++x) {
             uint4 v;
@@ -302,11 +311,12 @@ psrl_status_t dq_bf16(const AttnArgs& a) {
   p.Hq = P.Hq; p.G = P.Hq / P.Hkv; p.T_q = P.T_q;
   p.cap = cap; p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
   p.lse = a.lse_in; p.delta = a.delta; p.d_q = static_cast<__nv_bfloat16*>(a.d_q); p.status = a.status;
+  p.part = a.part;
   const int64_t grid = int64_t(P.q_tiles.size()) * P.Hq;
   if (grid > INT32_MAX) return PSRL_ERR_SHAPE;
   dq_kernel<<<unsigned(grid), kThreads, smem, a.stream>>>(m, p);
   if ((e = cudaGetLastError()) != cudaSuccess) return fail(e);
-  return PSRL_OK;
+  return merge_dq_bf16(a);
 }
 
 }  // namespace psrl

@@ -53,6 +53,8 @@ struct FwdParams {
   float scale_log2;
   __nv_bfloat16* o;
   float* lse;
+  float* part;      // partial rows [n_part_rows][Hq][128]: normalised O of items that do not own their rows
+  float* part_lse;  // [n_part_rows][Hq]
   int* status;
 };
 
@@ -201,7 +203,7 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
     for (int j = 0; j < n_tiles; ++j) {
       const int n_valid = nv_next;
       if (j + 1 < n_tiles) nv_next = path_nvalid[j + 1];
-      const bool diag = (j == n_tiles - 1);
+      const bool diag = qt.causal && (j == n_tiles - 1);
       const int limit = diag ? min(row + 1, n_valid) : n_valid;  // keys [0, limit) are visible
       const bool need_mask = diag || n_valid < 128;
       // ---- softmax of this tile: the whole score row in one round trip to tensor memory ----
@@ -283,12 +285,24 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       const float inv = 1.f / l_run;
       const bool store = row < qt.n_rows;
       const int h = h0 + q;
+      const bool partial = qt.part_row0 >= 0;
       __nv_bfloat16* orow = p.o + (int64_t(qt.q_row0 + row) * p.Hq + h) * 128;
+      float* prow = p.part + (int64_t(qt.part_row0 + row) * p.Hq + h) * 128;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
         tmem_ld32(t_lane + 128 + c * 32, r);
         tmem_wait_ld();
+        if (partial) {
+          if (store) {
+#pragma unroll
+            for (int x = 0; x < 8; ++x)
+              *reinterpret_cast<float4*>(prow + c * 32 + x * 4) =
+                  make_float4(__uint_as_float(r[4 * x]) * inv, __uint_as_float(r[4 * x + 1]) * inv,
+                              __uint_as_float(r[4 * x + 2]) * inv, __uint_as_float(r[4 * x + 3]) * inv);
+          }
+          continue;
+        }
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 32; i += 2)
@@ -299,6 +313,8 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
             *reinterpret_cast<uint4*>(orow + c * 32 + x * 8) = make_uint4(pk[4 * x], pk[4 * x + 1], pk[4 * x + 2], pk[4 * x + 3]);
         }
       }
+      if (store && partial) p.part_lse[int64_t(qt.part_row0 + row) * p.Hq + h] = (m_ref + log2f(l_run)) * kLn2;
+      else
       if (store) p.lse[int64_t(h) * p.T_q + qt.q_row0 + row] = (m_ref + log2f(l_run)) * kLn2;
     }
   }
@@ -340,6 +356,7 @@ psrl_status_t fwd_bf16(const AttnArgs& a) {
   p.scale_log2 = a.scale * kLog2e;
   p.o = static_cast<__nv_bfloat16*>(a.o_out);
   p.lse = a.lse_out;
+  p.part = a.part; p.part_lse = a.part_lse;
   p.status = a.status;
   const size_t smem = size_t(NQ + KS + VS) * kTileBytes + 1024;
   static bool attr_set = false;
@@ -354,7 +371,7 @@ psrl_status_t fwd_bf16(const AttnArgs& a) {
   fwd_kernel<<<unsigned(grid), kThreads, smem, a.stream>>>(maps, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_last_cuda_error(e); return PSRL_ERR_CUDA; }
-  return PSRL_OK;
+  return merge_fwd_bf16(a);
 }
 
 }  // namespace psrl

@@ -79,7 +79,7 @@ extern "C" psrl_status_t psrl_tree_attn_bwd_static(const psrl_plan_t* plan, cons
   if (!P.dev) return PSRL_ERR_WORKSPACE;  // plan not uploaded
   // the built-in scratch is a fixed size: larger problems must use psrl_tree_attn_bwd
   if (size_t(P.Hq) * size_t(P.T_q) > kMaxDeltaFloats) return PSRL_ERR_WORKSPACE;
-  if (psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P) + psrl::ws_slab_bytes(P) > kScratchBytes)
+  if (psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P) + psrl::ws_slab_bytes(P) + psrl::ws_part_bytes(P) > kScratchBytes)
     return PSRL_ERR_WORKSPACE;
   unsigned char* ws = static_cast<unsigned char*>(scratch_on_current_device());
   if (!ws) return PSRL_ERR_CUDA;
@@ -91,6 +91,7 @@ extern "C" psrl_status_t psrl_tree_attn_bwd_static(const psrl_plan_t* plan, cons
   a.status = reinterpret_cast<int*>(ws);
   a.delta = reinterpret_cast<float*>(ws + psrl::kWsHeaderBytes);
   a.slabs = reinterpret_cast<float*>(ws + psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P));
+  a.part = reinterpret_cast<float*>(ws + psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P) + psrl::ws_slab_bytes(P));
   a.pool_capacity = pool_capacity; a.scale = softmax_scale; a.stream = static_cast<cudaStream_t>(stream);
   // the array keeps the previous call's contents: the status header must start at zero;
   // D is fully rewritten by the pre-pass before anything reads it

@@ -6,8 +6,9 @@
 
 namespace psrl {
 
-// Layout of the caller's workspace: [0, 256) control words (word 0 = device
-// status), then D = rowsum(dO o O) as fp32 [Hq, T_q] for the backward.
+// Layout of the caller's workspace: [0, 256) control words (word 0 = device status), then
+//   forward:  partial O rows, their LSE
+//   backward: D = rowsum(dO o O) as fp32 [Hq, T_q], partial dV/dK slabs, partial dQ rows.
 constexpr size_t kWsHeaderBytes = 256;
 // After D: fp32 partial dV/dK slabs of split KV tiles, [slab][kv head][dV, dK][128][128].
 constexpr size_t kSlabBytes = size_t(2) * 128 * 128 * sizeof(float);
@@ -18,6 +19,16 @@ inline size_t ws_slab_bytes(const Plan& P) {
   return P.dtype == PSRL_BF16 ? size_t(P.n_slabs) * size_t(P.Hkv) * kSlabBytes : 0;
 }
 
+// Partial results of the forward / dQ items that do not own their rows (cascaded prefixes,
+// split-KV): fp32 [n_part_rows][Hq][128] (normalised O, or unscaled dQ), and for the
+// forward the parts' LSE as fp32 [n_part_rows][Hq] behind it.
+inline size_t ws_part_bytes(const Plan& P) {
+  return P.dtype == PSRL_BF16 ? size_t(P.n_part_rows) * size_t(P.Hq) * 128 * sizeof(float) : 0;
+}
+inline size_t ws_part_lse_bytes(const Plan& P) {
+  return P.dtype == PSRL_BF16 ? (size_t(P.n_part_rows) * size_t(P.Hq) * sizeof(float) + 255) / 256 * 256 : 0;
+}
+
 struct AttnArgs {
   const Plan* plan;
   const void *q, *k_pool, *v_pool, *o, *d_o;
@@ -26,6 +37,8 @@ struct AttnArgs {
   float* lse_out;
   float* delta;  // D, in the workspace
   float* slabs;  // partial dV/dK slabs, in the workspace (bf16 path)
+  float* part;   // partial O (forward) or dQ (backward) rows, in the workspace (bf16 path)
+  float* part_lse;  // LSE of the partial O rows (forward)
   int* status;   // device status word
   int64_t pool_capacity;
   float scale;
@@ -40,6 +53,8 @@ psrl_status_t fwd_bf16(const AttnArgs& a);
 psrl_status_t bwd_bf16(const AttnArgs& a);
 psrl_status_t dq_bf16(const AttnArgs& a);   // the dQ part of bwd_bf16
 psrl_status_t dkv_bf16(const AttnArgs& a);  // the dK/dV part of bwd_bf16 (+ reduce of split tiles)
+psrl_status_t merge_fwd_bf16(const AttnArgs& a);  // O, LSE of the rows assembled from partial results
+psrl_status_t merge_dq_bf16(const AttnArgs& a);   // dQ of those rows
 
 void set_last_cuda_error(cudaError_t e);
 

@@ -274,36 +274,66 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
         P.kv_tiles.push_back(kt);
       }
     }
-    // per-segment path of KV tiles and descendant query ranges
-    P.path_off.assign(n + 1, 0);
-    for (int32_t c = 0; c < n; ++c) {
-      int32_t cnt = P.seg_n_kvt[c];
-      for (int32_t i = P.anc_off[c]; i < P.anc_off[c + 1]; ++i) cnt += P.seg_n_kvt[P.anc_list[i]];
-      P.path_off[c + 1] = P.path_off[c] + cnt;
-    }
-    P.path_tiles.resize(P.path_off[n]);
+    // descendant query ranges (a subtree is a contiguous run of canonical indices)
     P.seg_desc_q_begin.assign(n, 0); P.seg_desc_q_end.assign(n, 0);
+    std::vector<int64_t> desc_qtiles(n, 0);  // own query tiles of all strict descendants
     for (int32_t c = 0; c < n; ++c) {
-      int32_t at = P.path_off[c];
-      auto emit = [&](int32_t seg) {
-        for (int32_t i = 0; i < P.seg_n_kvt[seg]; ++i) P.path_tiles[at++] = P.seg_first_kvt[seg] + i;
-      };
-      for (int32_t i = P.anc_off[c]; i < P.anc_off[c + 1]; ++i) emit(P.anc_list[i]);
-      emit(c);
       int32_t b = -1, e = -1;
       for (int32_t x = c + 1; x < P.seg_sub_end[c]; ++x) {
         if (P.seg_q_off[x] >= 0) {
           if (b < 0) b = P.seg_q_off[x];
           e = P.seg_q_off[x] + P.seg_len[x];
+          desc_qtiles[c] += P.seg_n_kvt[x];
         }
       }
       if (b >= 0) { P.seg_desc_q_begin[c] = b; P.seg_desc_q_end[c] = e; }
     }
-    // query tiles, longest first
+    // Which segments are cascaded (tensor-core path only).  Walking a's n_a KV tiles costs
+    // n_a tile steps per query tile that has a on its path: desc_qtiles[a] * n_a in total, or
+    // packed * n_a when the descendants' rows are packed 128 to a tile.  Cascade when packing
+    // at least halves that, or when the descendants' tiles are too few to occupy the SMs while
+    // a is long (the small-suffix / long-prefix case, which then also gets split over CTAs).
+    constexpr int64_t kSms = 148;
+    const int64_t cta_units = int64_t(P.Hkv) * ((P.Hq / P.Hkv + 1) / 2);  // forward CTAs per item
+    P.seg_cascaded.assign(n, 0);
+    if (P.dtype == PSRL_BF16) {
+      for (int32_t c = 0; c < n; ++c) {
+        const int64_t rows = P.seg_desc_q_end[c] - P.seg_desc_q_begin[c];
+        if (rows <= 0) continue;
+        const int64_t packed = (rows + kTile - 1) / kTile;
+        const bool fewer = packed * 2 <= desc_qtiles[c] && P.seg_n_kvt[c] >= 4;
+        const bool starved = desc_qtiles[c] * cta_units * 2 <= kSms && P.seg_n_kvt[c] >= 8;
+        P.seg_cascaded[c] = (fewer || starved) ? 1 : 0;
+      }
+    }
+    // per-segment list of KV tiles for the own items: non-cascaded ancestors root->parent, then own
+    P.path_off.assign(n + 1, 0);
+    std::vector<uint8_t> has_casc_anc(n, 0);
+    for (int32_t c = 0; c < n; ++c) {
+      int32_t cnt = P.seg_n_kvt[c];
+      for (int32_t i = P.anc_off[c]; i < P.anc_off[c + 1]; ++i) {
+        const int32_t a = P.anc_list[i];
+        if (P.seg_cascaded[a]) has_casc_anc[c] = 1; else cnt += P.seg_n_kvt[a];
+      }
+      P.path_off[c + 1] = P.path_off[c] + cnt;
+    }
+    P.path_tiles.resize(P.path_off[n]);
+    for (int32_t c = 0; c < n; ++c) {
+      int32_t at = P.path_off[c];
+      auto emit = [&](int32_t seg) {
+        for (int32_t i = 0; i < P.seg_n_kvt[seg]; ++i) P.path_tiles[at++] = P.seg_first_kvt[seg] + i;
+      };
+      for (int32_t i = P.anc_off[c]; i < P.anc_off[c + 1]; ++i)
+        if (!P.seg_cascaded[P.anc_list[i]]) emit(P.anc_list[i]);
+      emit(c);
+    }
+    // own items
     P.qrow_seg.resize(P.T_q);
+    std::vector<int32_t> own_part_base(n, -1);
     for (int32_t c = 0; c < n; ++c) {
       if (P.seg_q_off[c] < 0) continue;
       for (int32_t i = 0; i < P.seg_len[c]; ++i) P.qrow_seg[P.seg_q_off[c] + i] = c;
+      if (has_casc_anc[c]) { own_part_base[c] = P.n_part_rows; P.n_part_rows += P.seg_len[c]; }
       const int32_t anc_tiles = (P.path_off[c + 1] - P.path_off[c]) - P.seg_n_kvt[c];
       for (int32_t t = 0; t < P.seg_n_kvt[c]; ++t) {
         QTile qt{};
@@ -313,7 +343,57 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
         qt.n_rows = std::min(kTile, P.seg_len[c] - t * kTile);
         qt.pt_begin = P.path_off[c];
         qt.n_kv_tiles = anc_tiles + t + 1;
+        qt.causal = 1;
+        qt.part_row0 = has_casc_anc[c] ? own_part_base[c] + t * kTile : -1;
         P.q_tiles.push_back(qt);
+      }
+    }
+    // packed items of the cascaded segments: chunk k of a's tiles x block b of 128 packed rows;
+    // partial rows of chunk k are [base + k*rows, base + (k+1)*rows), in query-row order
+    std::vector<int32_t> casc_part_base(n, -1), casc_chunks(n, 0);
+    for (int32_t a = 0; a < n; ++a) {
+      if (!P.seg_cascaded[a]) continue;
+      const int32_t rows = P.seg_desc_q_end[a] - P.seg_desc_q_begin[a];
+      const int32_t packed = (rows + kTile - 1) / kTile, nt = P.seg_n_kvt[a];
+      int64_t chunks = (kSms + packed * cta_units - 1) / (packed * cta_units);
+      chunks = std::max<int64_t>(1, std::min<int64_t>(chunks, nt / 2));
+      casc_part_base[a] = P.n_part_rows;
+      casc_chunks[a] = static_cast<int32_t>(chunks);
+      for (int32_t k = 0; k < chunks; ++k) {
+        const int32_t t0 = static_cast<int32_t>(int64_t(nt) * k / chunks), t1 = static_cast<int32_t>(int64_t(nt) * (k + 1) / chunks);
+        const int32_t pt = static_cast<int32_t>(P.path_tiles.size());
+        for (int32_t t = t0; t < t1; ++t) P.path_tiles.push_back(P.seg_first_kvt[a] + t);
+        for (int32_t b = 0; b < packed; ++b) {
+          QTile qt{};
+          qt.seg = a;
+          qt.tile_idx = k;
+          qt.q_row0 = P.seg_desc_q_begin[a] + b * kTile;
+          qt.n_rows = std::min(kTile, rows - b * kTile);
+          qt.pt_begin = pt;
+          qt.n_kv_tiles = t1 - t0;
+          qt.causal = 0;
+          qt.part_row0 = P.n_part_rows + k * rows + b * kTile;
+          P.q_tiles.push_back(qt);
+        }
+      }
+      P.n_part_rows += static_cast<int32_t>(chunks) * rows;
+    }
+    // merge lists: cascaded ancestors root->parent (chunks ascending), then the own item
+    P.merge_off.push_back(0);
+    for (int32_t c = 0; c < n; ++c) {
+      if (P.seg_q_off[c] < 0 || !has_casc_anc[c]) continue;
+      for (int32_t i = 0; i < P.seg_len[c]; ++i) {
+        const int32_t r = P.seg_q_off[c] + i;
+        P.merge_row.push_back(r);
+        for (int32_t x = P.anc_off[c]; x < P.anc_off[c + 1]; ++x) {
+          const int32_t a = P.anc_list[x];
+          if (!P.seg_cascaded[a]) continue;
+          const int32_t rows = P.seg_desc_q_end[a] - P.seg_desc_q_begin[a];
+          for (int32_t k = 0; k < casc_chunks[a]; ++k)
+            P.merge_parts.push_back(casc_part_base[a] + k * rows + (r - P.seg_desc_q_begin[a]));
+        }
+        P.merge_parts.push_back(own_part_base[c] + i);
+        P.merge_off.push_back(static_cast<int32_t>(P.merge_parts.size()));
       }
     }
     std::stable_sort(P.q_tiles.begin(), P.q_tiles.end(),
@@ -349,7 +429,7 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
       total_sub += it.sub_end;
       whole.push_back(it);
     }
-    constexpr int64_t kSms = 148, kMinPart = 12;
+    constexpr int64_t kMinPart = 12;
     const int64_t fair = (total_sub * P.Hkv + kSms - 1) / kSms;       // sub-tiles per SM if perfectly balanced
     const int64_t part_max = std::max<int64_t>(kMinPart, fair / 2);
     for (const KvItem& it : whole) {
@@ -412,6 +492,11 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
     H.off_split = append_array(B, P.kv_splits);
     H.n_split = static_cast<int32_t>(P.kv_splits.size());
     H.n_slabs = P.n_slabs;
+    H.n_part_rows = P.n_part_rows;
+    H.n_merge_rows = static_cast<int32_t>(P.merge_row.size());
+    H.off_merge_row = append_array(B, P.merge_row);
+    H.off_merge_off = append_array(B, P.merge_off);
+    H.off_merge_parts = append_array(B, P.merge_parts);
     while (B.size() % 64) B.push_back(0);
     std::copy(reinterpret_cast<const int32_t*>(&H), reinterpret_cast<const int32_t*>(&H + 1), B.begin());
   } catch (const std::bad_alloc&) {

@@ -26,15 +26,29 @@ struct KvTile {
   int32_t pad0, pad1, pad2;
 };
 
-// One query tile: up to 128 consecutive rows of one HAS_Q segment.
+// One work item of the forward and dQ kernels: up to 128 consecutive query rows
+// and a list of KV tiles they attend to.
+//  * own item: rows of one HAS_Q segment; the list holds the tiles of its
+//    ancestors root->parent (those that are not cascaded, see below) and its own
+//    tiles up to the diagonal tile, which is last and causal.
+//  * packed item: rows of the contiguous query range of ALL strict descendants of
+//    a "cascaded" segment a (rows of several short segments share one tile) and a
+//    chunk of a's KV tiles, every key visible to every row.  A segment is cascaded
+//    when its descendants' own tiles are mostly empty or too few to fill the GPU;
+//    its KV tiles are then visited once per 128 packed rows instead of once per
+//    descendant tile, and split into chunks over CTAs (split-KV).
+// An item whose rows also get contributions from other items writes fp32 partial
+// results to rows [part_row0, part_row0 + n_rows) of the workspace; the merge
+// kernels combine the parts of a row in the fixed order of its merge list.
 struct QTile {
-  int32_t seg;
-  int32_t tile_idx;   // rows [tile_idx*128, ...) of the segment
+  int32_t seg;        // segment of the rows (own item) or the cascaded ancestor (packed item)
+  int32_t tile_idx;   // own item: rows [tile_idx*128, ...) of the segment; packed item: chunk index
   int32_t q_row0;     // first row in Q/O/dO/dQ
   int32_t n_rows;     // 1..128
-  int32_t pt_begin;   // range in path_tiles: ancestors' tiles root->parent, then own tiles 0..tile_idx
-  int32_t n_kv_tiles; // tiles to visit; the last one is the diagonal tile
-  int32_t pad0, pad1;
+  int32_t pt_begin;   // first entry in path_tiles
+  int32_t n_kv_tiles; // tiles to visit
+  int32_t causal;     // 1: the last tile is the diagonal tile of the rows' segment; 0: every key visible
+  int32_t part_row0;  // -1: the item writes the final outputs; else its first partial row
 };
 
 constexpr int kSubRows = 128;  // query rows per step of the dK/dV kernel
@@ -72,7 +86,10 @@ struct DeviceHeader {
   int32_t off_path_nvalid;  // valid keys of every entry of path_tiles
   int32_t n_kvi;
   int32_t n_split, off_split, n_slabs;
-  int32_t reserved[3];
+  // merge lists of the rows that are assembled from partial results: row i of the list is
+  // query row merge_row[i]; its parts are merge_parts[merge_off[i] .. merge_off[i+1]) (partial-row ids)
+  int32_t n_part_rows, n_merge_rows, off_merge_row, off_merge_off, off_merge_parts;
+  int32_t reserved[2];
 };
 
 struct Plan {
@@ -93,6 +110,9 @@ struct Plan {
   std::vector<KvItem> kv_items;  // longest first
   std::vector<KvSplit> kv_splits;
   int32_t n_slabs = 0;
+  std::vector<uint8_t> seg_cascaded;  // 1: the segment's KV tiles are handled by packed items
+  int32_t n_part_rows = 0;
+  std::vector<int32_t> merge_row, merge_off, merge_parts;
   std::vector<int32_t> seg_first_kvt, seg_n_kvt, seg_desc_q_begin, seg_desc_q_end, path_off, path_tiles, path_nvalid, qrow_seg;
   // device blob
   std::vector<int32_t> blob;

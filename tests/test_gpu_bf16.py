@@ -96,9 +96,45 @@ def test_reduced_configs(lib, name, scale_len):
     check(lib, w, seed=100)
 
 
+def test_small_suffixes_on_a_long_prefix(lib):
+    """The memory-bound case: a cached prefix (no queries) and suffixes of a few tokens.  The
+    prefix's KV tiles are visited by packed rows and split over CTAs; rows are assembled by
+    the merge kernels (forward: log-sum-exp of the parts, backward: sum of the parts' dQ)."""
+    flags = [0] + [3] * 8
+    w = Workload("ss", [-1] + [0] * 8, [1100, 1, 2, 3, 4, 5, 6, 7, 8], [64], 8, 2, 128, "bf16", seg_flags=flags)
+    plan, _, _ = check(lib, w, seed=40)
+    assert lib.psrl_launch_count(plan, False) == 2
+    # the same with queries on the prefix, G = 3 (a head pair + a single head)
+    check(lib, Workload("ssq", [-1] + [0] * 8, [1100, 1, 2, 3, 4, 5, 6, 7, 8], [32], 6, 2, 128, "bf16"), seed=41)
+    # full-size c2s
+    w = make_workload("c2s", 3)
+    plan, _, _ = check(lib, w, seed=42)
+    assert lib.psrl_launch_count(plan, False) == 2
+
+
+def test_nested_cascades(lib):
+    """Two levels of long segments above many short leaves: rows merge the parts of two
+    cascaded ancestors and their own item; more than 128 packed rows (two row blocks)."""
+    parent, seg_len = [-1, 0, 0, 0], [600, 520, 9, 11]
+    for _ in range(30):
+        parent.append(1)
+        seg_len.append(5)
+    plan, _, _ = check(lib, Workload("nest", parent, seg_len, [128], 4, 2, 128, "bf16"), seed=43)
+    assert lib.psrl_launch_count(plan, True) >= 4
+
+
 def test_runs_are_bitwise_reproducible(lib):
     w = Workload("det", [-1, 0, 0, 1], [700, 300, 129, 50], [64], 8, 2, 128, "bf16")
     plan, (q, k, v, d_o), a = check(lib, w, seed=12)
+    for _ in range(2):
+        b = run_gpu(lib, plan, q, k, v, d_o, w.softmax_scale)
+        for key in ("O", "LSE", "dQ"):
+            assert torch.equal(a[key], b[key])
+        for key in ("dK", "dV"):
+            assert torch.equal(torch.nan_to_num(a[key]), torch.nan_to_num(b[key]))
+    # and with merged rows (cascaded prefix, split over CTAs)
+    w = make_workload("c2s", 5)
+    plan, (q, k, v, d_o), a = check(lib, w, seed=13)
     for _ in range(2):
         b = run_gpu(lib, plan, q, k, v, d_o, w.softmax_scale)
         for key in ("O", "LSE", "dQ"):
