@@ -316,6 +316,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
     const int wg = warp >> 2;                            // which 64 query columns of the 128
     const int keyrow = (warp & 3) * 32 + lane;           // key inside the tile = TMEM lane
     const uint32_t t_lane = tmem + (uint32_t((warp & 3) * 32) << 16);
+    const f32x2 scale2 = make_f32x2(p.scale_log2, p.scale_log2);
     bool ok = true;
     for (int i = 0; i < n_it; ++i) {
       int g, row0, nvq, qpos0; bool diag;
@@ -336,8 +337,9 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
           uint32_t pk[16];
 #pragma unroll
           for (int x = 0; x < 32; x += 2) {
-            float p0 = ex2(__uint_as_float(s[c][x]) * p.scale_log2);
-            float p1 = ex2(__uint_as_float(s[c][x + 1]) * p.scale_log2);
+            float a0, a1;
+            split_f32x2(mul2(make_f32x2(s[c][x], s[c][x + 1]), scale2), a0, a1);
+            float p0 = ex2(a0), p1 = ex2(a1);
             if (diag) {  // the tile that holds the keys' own rows: a key is visible from its own row on
               const int col = wg * 64 + c * 32 + x;
               p0 = (qpos0 + col >= keyrow) ? p0 : 0.f;
@@ -366,9 +368,11 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
         for (int c = 0; c < 2; ++c) {
           uint32_t pk[16];
 #pragma unroll
-          for (int x = 0; x < 32; x += 2)
-            pk[x >> 1] = pack_bf16(pr[c * 32 + x] * __uint_as_float(dp[c][x]),
-                                   pr[c * 32 + x + 1] * __uint_as_float(dp[c][x + 1]));
+          for (int x = 0; x < 32; x += 2) {
+            float d0, d1;
+            split_f32x2(mul2(make_f32x2(pr[c * 32 + x], pr[c * 32 + x + 1]), make_f32x2(dp[c][x], dp[c][x + 1])), d0, d1);
+            pk[x >> 1] = pack_bf16(d0, d1);
+          }
           tmem_st16(t_lane + TM_DPT + wg * 64 + c * 16, pk);
         }
       }

@@ -10,14 +10,16 @@
 // dQ accumulates in tensor memory over the whole path, so every dQ row is
 // summed in path order by one CTA (bitwise reproducible).
 //
-// The warps work in two half-steps so that the tensor cores never wait for a
-// whole softmax: S may be overwritten as soon as the warps have READ it (P is
-// not stored back), so S(j+1) is issued while P(j) is still being computed;
-// dP(j+1) is issued right after dQ(j), which consumed dS(j).
+// The tensor cores run one step ahead of the warps: S may be overwritten as
+// soon as the warps have READ it into registers (P is never stored), so S(j+1)
+// is issued while step j is still being computed; dP / dS has two buffers, so
+// dP(j+1) follows right behind S(j+1).  The warps therefore find both inputs of
+// a step ready, fetch them in one tensor-memory round trip and compute P and dS
+// element by element in one pass.
 //
 // Warp roles: warps 0-7 softmax-backward (two threads per query row, 64 keys
 // each), warp 8 TMA producer, warp 9 MMA issuer + TMEM owner.
-// Tensor memory: S at 0, dP / dS at 128, dQ at 256.
+// Tensor memory: S at 0, dP / dS at 128 and 256 (alternating), dQ at 384.
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -31,7 +33,7 @@ using namespace sm100;
 
 constexpr int KS = 3, VS = 2;                 // K and V ring depths
 constexpr int kThreads = (8 + 2) * 32;
-constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 256;
+constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 384;   // dP / dS is double-buffered: 128 and 256
 
 struct Maps {
   CUtensorMap q, d_o;
@@ -51,7 +53,7 @@ struct Params {
 };
 struct __align__(8) Barriers {
   uint64_t qdo_full, k_full[KS], k_empty[KS], v_full[VS], v_empty[VS];
-  uint64_t s_full, s_free, dp_full, ds_ready, dq_done;
+  uint64_t s_full, s_free, dp_full[2], ds_ready[2], dq_done;
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -79,7 +81,7 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     for (int i = 0; i < KS; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1); }
     for (int i = 0; i < VS; ++i) { mbar_init(&bar.v_full[i], 1); mbar_init(&bar.v_empty[i], 1); }
     mbar_init(&bar.s_full, 1); mbar_init(&bar.s_free, 256);
-    mbar_init(&bar.dp_full, 1); mbar_init(&bar.ds_ready, 256);
+    for (int i = 0; i < 2; ++i) { mbar_init(&bar.dp_full[i], 1); mbar_init(&bar.ds_ready[i], 256); }
     mbar_init(&bar.dq_done, 1);
     fence_mbar_init();
   }
@@ -136,38 +138,37 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       mma_kk(tmem + TM_S, q_lo, k_lo);
       commit(&bar.s_full);
       mma_kk(tmem + TM_DP, g_lo, v_lo);
-      commit(&bar.dp_full);
+      commit(&bar.dp_full[0]);
       commit(&bar.v_empty[0]);
     }
     for (int j = 0; ok && j < n_tiles; ++j) {
       if (j + 1 < n_tiles) {
-        ok = wait(&bar.k_full[(j + 1) % KS], ((j + 1) / KS) & 1) && wait(&bar.s_free, j & 1);
+        // S(j+1) as soon as the warps have read S(j); dP(j+1) into the other dP buffer (last read
+        // by dQ(j-1), which precedes it in the tensor pipe), so the warps' next step finds both ready
+        const int vs = (j + 1) % VS;
+        ok = mbar_wait_all3(&bar.k_full[(j + 1) % KS], ((j + 1) / KS) & 1, &bar.v_full[vs], ((j + 1) / VS) & 1,
+                            &bar.s_free, j & 1, abortp, p.status);
         if (!ok) break;
         tc_fence_after();
         mma_kk(tmem + TM_S, q_lo, k_lo + ((j + 1) % KS) * (kTileBytes >> 4));
         commit(&bar.s_full);
+        mma_kk(tmem + TM_DP + ((j + 1) & 1) * 128, g_lo, v_lo + vs * (kTileBytes >> 4));
+        commit(&bar.dp_full[(j + 1) & 1]);
+        commit(&bar.v_empty[vs]);
       }
-      ok = wait(&bar.ds_ready, j & 1);
+      ok = mbar_wait_all1(&bar.ds_ready[j & 1], (j >> 1) & 1, abortp, p.status);
       if (!ok) break;
       tc_fence_after();
       if (elect_one()) {
         // dS: packed bf16, 16 keys per 8 columns; keys 0-63 at +0, keys 64-127 at +64
         const uint32_t b0 = k_mn + (j % KS) * (kTileBytes >> 4);
+        const uint32_t a0 = tmem + TM_DP + (j & 1) * 128;
         const uint32_t acc0 = j > 0;
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-          mma_ts_lo(tmem + TM_DQ, tmem + TM_DP + (k >> 2) * 64 + (k & 3) * 8, b0 + k * 128, idesc_mn,
-                    k > 0 ? 1u : acc0);
+          mma_ts_lo(tmem + TM_DQ, a0 + (k >> 2) * 64 + (k & 3) * 8, b0 + k * 128, idesc_mn, k > 0 ? 1u : acc0);
       }
       commit(&bar.k_empty[j % KS]);
-      if (j + 1 < n_tiles) {
-        const int vs = (j + 1) % VS;
-        ok = wait(&bar.v_full[vs], ((j + 1) / VS) & 1);
-        if (!ok) break;
-        mma_kk(tmem + TM_DP, g_lo, v_lo + vs * (kTileBytes >> 4));
-        commit(&bar.dp_full);
-        commit(&bar.v_empty[vs]);
-      }
     }
     if (ok) commit(&bar.dq_done);
   } else {
@@ -178,6 +179,8 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     const bool row_ok = row < qt.n_rows;
     const float lse2 = row_ok ? p.lse[int64_t(h) * p.T_q + qt.q_row0 + row] * kLog2e : 0.f;
     const float dl = row_ok ? p.delta[int64_t(h) * p.T_q + qt.q_row0 + row] : 0.f;
+    const f32x2 scale2 = make_f32x2(p.scale_log2, p.scale_log2), neg_lse2 = make_f32x2(-lse2, -lse2),
+                neg_dl2 = make_f32x2(-dl, -dl);
     bool ok = true;
     int nv_next = path_nvalid[0];
     for (int j = 0; j < n_tiles; ++j) {
@@ -186,51 +189,39 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       const bool diag = qt.causal && (j == n_tiles - 1);
       const int limit = diag ? min(row + 1, n_valid) : n_valid;   // keys [0, limit) are visible
       const bool need_mask = diag || n_valid < 128;
-      float pr[64];
-      // ---- half-step 1: read S, release it, P = exp2(S c - LSE) ----
-      ok = mbar_wait(&bar.s_full, j & 1, abortp, p.status);
+      // S(j) and dP(j) are both complete well before the warps get here (the MMA warp issues them
+      // one step ahead), so both are fetched in one round trip; S may then be overwritten.
+      const uint32_t t_dp = t_lane + TM_DP + (j & 1) * 128;
+      ok = mbar_wait(&bar.s_full, j & 1, abortp, p.status) &&
+           mbar_wait(&bar.dp_full[j & 1], (j >> 1) & 1, abortp, p.status);
       if (!ok) break;
       tc_fence_after();
-      {
-        uint32_t s[2][32];
-        tmem_ld32(t_lane + TM_S + half * 64, s[0]);
-        tmem_ld32(t_lane + TM_S + half * 64 + 32, s[1]);
-        tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(&bar.s_free);
+      uint32_t s[2][32], dp[2][32];
+      tmem_ld32(t_lane + TM_S + half * 64, s[0]);
+      tmem_ld32(t_lane + TM_S + half * 64 + 32, s[1]);
+      tmem_ld32(t_dp + half * 64, dp[0]);
+      tmem_ld32(t_dp + half * 64 + 32, dp[1]);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(&bar.s_free);
+      // P = exp2(S c - LSE) and dS = P o (dP - D) element by element: the exp2 (MUFU pipe) of one
+      // element overlaps the arithmetic of its neighbours instead of forming a phase of its own
 #pragma unroll
-        for (int c = 0; c < 2; ++c)
+      for (int c = 0; c < 2; ++c) {
+        uint32_t pk[16];
 #pragma unroll
-          for (int x = 0; x < 32; ++x) {
-            float pv = ex2(fmaf(__uint_as_float(s[c][x]), p.scale_log2, -lse2));
-            if (need_mask) pv = (half * 64 + c * 32 + x < limit) ? pv : 0.f;
-            pr[c * 32 + x] = pv;
+        for (int x = 0; x < 32; x += 2) {
+          float a0, a1, d0, d1;
+          split_f32x2(fma2(make_f32x2(s[c][x], s[c][x + 1]), scale2, neg_lse2), a0, a1);
+          const f32x2 pp = make_f32x2(ex2(a0), ex2(a1));
+          split_f32x2(mul2(pp, add2(make_f32x2(dp[c][x], dp[c][x + 1]), neg_dl2)), d0, d1);
+          if (need_mask) {  // masked columns may hold anything (pad rows of K, V): select, do not multiply
+            d0 = (half * 64 + c * 32 + x < limit) ? d0 : 0.f;
+            d1 = (half * 64 + c * 32 + x + 1 < limit) ? d1 : 0.f;
           }
-      }
-      // ---- half-step 2: dS = P o (dP - D) ----
-      ok = mbar_wait(&bar.dp_full, j & 1, abortp, p.status);
-      if (!ok) break;
-      tc_fence_after();
-      {
-        uint32_t dp[2][32];
-        tmem_ld32(t_lane + TM_DP + half * 64, dp[0]);
-        tmem_ld32(t_lane + TM_DP + half * 64 + 32, dp[1]);
-        tmem_wait_ld();
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int x = 0; x < 32; x += 2) {
-            float d0 = pr[c * 32 + x] * (__uint_as_float(dp[c][x]) - dl);
-            float d1 = pr[c * 32 + x + 1] * (__uint_as_float(dp[c][x + 1]) - dl);
-            if (need_mask) {  // masked columns may hold anything (pad rows of V): select, do not multiply
-              d0 = (half * 64 + c * 32 + x < limit) ? d0 : 0.f;
-              d1 = (half * 64 + c * 32 + x + 1 < limit) ? d1 : 0.f;
-            }
-            pk[x >> 1] = pack_bf16(d0, d1);
-          }
-          tmem_st16(t_lane + TM_DP + half * 64 + c * 16, pk);
+          pk[x >> 1] = pack_bf16(d0, d1);
         }
+        tmem_st16(t_dp + half * 64 + c * 16, pk);
       }
       // K rows at or beyond n_valid must be zero before dS K (dS is zero there, K may hold anything)
       if (n_valid < 128 && half == 0) {
@@ -241,7 +232,7 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       }
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bar.ds_ready);
+      mbar_arrive(&bar.ds_ready[j & 1]);
     }
     // ---- dQ = scale * accumulator ----
     if (ok) ok = mbar_wait(&bar.dq_done, 0, abortp, p.status);

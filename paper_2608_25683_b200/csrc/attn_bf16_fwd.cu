@@ -198,6 +198,7 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
     // the maximum has grown by more than 2^8, so the output accumulator in tensor memory
     // is rescaled rarely (typically only on the first tiles) instead of once per tile.
     float m_ref = -CUDART_INF_F, l_run = 0.f;
+    const f32x2 scale2 = make_f32x2(p.scale_log2, p.scale_log2);
     bool ok = true;
     int nv_next = path_nvalid[0];
     for (int j = 0; j < n_tiles; ++j) {
@@ -233,23 +234,28 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       const bool any_move = __any_sync(0xffffffffu, move);
       const float m_use = move ? m_new : m_ref;
       const float alpha = ex2(m_ref - m_use);            // 1 if the reference stays, 0 on the first tile
-      float sum = 0.f;
+      f32x2 sum2 = make_f32x2(0.f, 0.f);
+      const f32x2 neg_m2 = make_f32x2(-m_use, -m_use);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t pk[16];
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
-          float e0 = ex2(fmaf(__uint_as_float(s[c][i]), p.scale_log2, -m_use));
-          float e1 = ex2(fmaf(__uint_as_float(s[c][i + 1]), p.scale_log2, -m_use));
+          float a0, a1;
+          split_f32x2(fma2(make_f32x2(s[c][i], s[c][i + 1]), scale2, neg_m2), a0, a1);
+          float e0 = ex2(a0), e1 = ex2(a1);
           if (need_mask) {
             e0 = (c * 32 + i < limit) ? e0 : 0.f;
             e1 = (c * 32 + i + 1 < limit) ? e1 : 0.f;
           }
-          sum += e0 + e1;
+          sum2 = add2(sum2, make_f32x2(e0, e1));
           pk[i >> 1] = pack_bf16(e0, e1);
         }
         tmem_st16(t_lane + c * 16, pk);
       }
+      float sum_lo, sum_hi;
+      split_f32x2(sum2, sum_lo, sum_hi);
+      const float sum = sum_lo + sum_hi;
       l_run = fmaf(l_run, alpha, sum);
       m_ref = m_use;
       // ---- the reference moved: rescale the accumulated output in tensor memory ----

@@ -88,6 +88,52 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity
   return false;
 }
 
+// Non-blocking test of a phase, relaxed ordering (see mbar_wait_relaxed for why that is enough
+// for the MMA-issuing warp).
+__device__ __forceinline__ bool mbar_test_relaxed(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.relaxed.cta.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait of the MMA-issuing warp on up to three barriers at once.  A wait costs that warp
+// 100-350 cycles even when the phase is already complete (the barrier lives in shared memory,
+// whose pipeline the running MMAs keep busy), and the tensor pipe queues only a few MMAs, so every
+// separate wait between two groups of MMAs opens a bubble.  Testing the barriers side by side
+// costs one such latency instead of three.  All lanes take part (warp-uniform result).
+__device__ __forceinline__ bool mbar_wait_all3(uint64_t* b0, uint32_t p0, uint64_t* b1, uint32_t p1, uint64_t* b2,
+                                               uint32_t p2, volatile int* s_abort, int* g_status) {
+  bool d0 = false, d1 = false, d2 = false;
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    const bool t0 = d0 || mbar_test_relaxed(b0, p0);
+    const bool t1 = d1 || mbar_test_relaxed(b1, p1);
+    const bool t2 = d2 || mbar_test_relaxed(b2, p2);
+    d0 = t0; d1 = t1; d2 = t2;
+    if (__all_sync(0xffffffffu, d0 && d1 && d2)) return true;
+    if (it > 1024 && *s_abort) return false;
+  }
+  *s_abort = 1;
+  if (g_status) atomicExch(g_status, 10);
+  return false;
+}
+
+// The same for one barrier.
+__device__ __forceinline__ bool mbar_wait_all1(uint64_t* b0, uint32_t p0, volatile int* s_abort, int* g_status) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (__all_sync(0xffffffffu, mbar_test_relaxed(b0, p0))) return true;
+    if (it > 1024 && *s_abort) return false;
+  }
+  *s_abort = 1;
+  if (g_status) atomicExch(g_status, 10);
+  return false;
+}
+
 // One lane of a fully active warp (the same lane every time for the same mask).
 // Issuing tcgen05 instructions under this predicate, inside warp-uniform control
 // flow, measured ~40 % more MMA throughput than a `lane == 0` branch when the
@@ -256,6 +302,41 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// Packed fp32 pairs (sm_100 executes two fp32 operations per instruction on a 64-bit register
+// pair): the softmax warps are bound by instruction issue, and every slot they free goes to the
+// MMA-issuing warp that shares their scheduler.
+struct f32x2 {
+  uint64_t v;
+};
+__device__ __forceinline__ f32x2 make_f32x2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ f32x2 make_f32x2(uint32_t lo, uint32_t hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void split_f32x2(f32x2 a, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a.v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v));
+  return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+  return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+  return r;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
