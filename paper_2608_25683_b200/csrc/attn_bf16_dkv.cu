@@ -294,6 +294,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
         tc_fence_after();
         mma_acc(tmem + TM_DV, tmem + TM_ST, g_mn + so, i > 0);
         if (i + 1 < n_it) {
+          // the Q / dO tiles of step i+1 arrive late (two-stage ring): wait behind dV(i), not before it
           ok = wait(&bar.qd_full[(i + 1) % ST], ((i + 1) / ST) & 1);
           if (!ok) break;
           mma_kk(tmem + TM_ST, k_lo, q_lo + so1, lsex_lo + sx1);

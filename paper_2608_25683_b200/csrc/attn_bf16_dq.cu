@@ -98,6 +98,8 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       mbar_expect_tx(&bar.qdo_full, 2 * kTileBytes);
       load_row_tile(sQ, &maps.q, &bar.qdo_full, h, qt.q_row0);
       load_row_tile(sdO, &maps.d_o, &bar.qdo_full, h, qt.q_row0);
+    }
+    if (lane == 0) {
       const KvTile* kvt = reinterpret_cast<const KvTile*>(p.blob + p.off_kvt);
       const int32_t* page_slot = p.blob + p.off_page_slot;
       const int64_t head_row0 = int64_t(hk) * p.cap;
@@ -146,8 +148,8 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
         // S(j+1) as soon as the warps have read S(j); dP(j+1) into the other dP buffer (last read
         // by dQ(j-1), which precedes it in the tensor pipe), so the warps' next step finds both ready
         const int vs = (j + 1) % VS;
-        ok = mbar_wait_all3(&bar.k_full[(j + 1) % KS], ((j + 1) / KS) & 1, &bar.v_full[vs], ((j + 1) / VS) & 1,
-                            &bar.s_free, j & 1, abortp, p.status);
+        ok = mbar_wait_all3(&bar.s_free, j & 1, &bar.k_full[(j + 1) % KS], ((j + 1) / KS) & 1, &bar.v_full[vs],
+                            ((j + 1) / VS) & 1, abortp, p.status);
         if (!ok) break;
         tc_fence_after();
         mma_kk(tmem + TM_S, q_lo, k_lo + ((j + 1) % KS) * (kTileBytes >> 4));

@@ -113,6 +113,8 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       for (int q = 0; q < nq; ++q) {
         load_row_tile(sQ + q * kTileBytes, &maps.q, &bar.q_full, h0 + q, qt.q_row0);
       }
+    }
+    if (lane == 0) {
       const KvTile* kvt = reinterpret_cast<const KvTile*>(p.blob + p.off_kvt);
       const int32_t* page_slot = p.blob + p.off_page_slot;
       const int64_t head_row0 = int64_t(hk) * p.cap;
@@ -169,8 +171,17 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       for (int j = 0; ok && j < n_tiles; ++j) {
         const int vs = j % VS;
         for (int q = 0; ok && q < nq; ++q) {
-          ok = wait(&bar.p_ready[q], j & 1);
-          if (ok && q == 0) ok = wait(&bar.v_full[vs], (j / VS) & 1);
+          // one round of barrier tests per head: for head 0 also the V tile of this step and the K tile
+          // of the next one (each separate wait would cost the issuing warp hundreds of cycles)
+          if (q == 0) {
+            const bool more = j + 1 < n_tiles;
+            const int ksn = (j + 1) % KS;
+            ok = mbar_wait_all3(&bar.p_ready[0], j & 1, &bar.v_full[vs], (j / VS) & 1,
+                                more ? &bar.k_full[ksn] : &bar.v_full[vs], more ? ((j + 1) / KS) & 1 : (j / VS) & 1,
+                                abortp, p.status);
+          } else {
+            ok = mbar_wait_all1(&bar.p_ready[q], j & 1, abortp, p.status);
+          }
           if (!ok) break;
           tc_fence_after();
           issue_pv(q, vs, j == 0);
@@ -178,9 +189,6 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
           if (q == nq - 1) commit(&bar.v_empty[vs]);
           if (j + 1 < n_tiles) {
             const int ks = (j + 1) % KS;
-            if (q == 0) ok = wait(&bar.k_full[ks], ((j + 1) / KS) & 1);
-            if (!ok) break;
-            tc_fence_after();
             issue_s(q, ks);
             commit(&bar.s_full[q]);
             if (q == nq - 1) commit(&bar.k_empty[ks]);
@@ -227,7 +235,7 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
         for (int c = 0; c < 4; ++c)
 #pragma unroll
           for (int i = 0; i < 32; i += 2)
-            mx = fmaxf(mx, fmaxf(__uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1])));
+            mx = fmax3(mx, __uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1]));
       }
       const float m_new = fmaxf(m_ref, mx * p.scale_log2);
       const bool move = m_new > m_ref + 8.f;            // also true on the first tile (m_ref = -inf)

@@ -104,18 +104,18 @@ __device__ __forceinline__ bool mbar_test_relaxed(uint64_t* bar, uint32_t parity
 
 // Bounded wait of the MMA-issuing warp on up to three barriers at once.  A wait costs that warp
 // 100-350 cycles even when the phase is already complete (the barrier lives in shared memory,
-// whose pipeline the running MMAs keep busy), and the tensor pipe queues only a few MMAs, so every
-// separate wait between two groups of MMAs opens a bubble.  Testing the barriers side by side
-// costs one such latency instead of three.  All lanes take part (warp-uniform result).
+// whose pipeline the running MMAs keep busy, and the warp competes with the softmax warps for
+// issue slots), and the tensor pipe queues only a few MMAs, so every separate wait between two
+// groups of MMAs opens a bubble.  The first barrier is the one expected to complete last: the warp
+// blocks on it with try_wait (suspended by the hardware, no issue slots taken from the softmax
+// warps), then tests the other two side by side.  All lanes take part (warp-uniform result).
 __device__ __forceinline__ bool mbar_wait_all3(uint64_t* b0, uint32_t p0, uint64_t* b1, uint32_t p1, uint64_t* b2,
                                                uint32_t p2, volatile int* s_abort, int* g_status) {
-  bool d0 = false, d1 = false, d2 = false;
+  if (!__all_sync(0xffffffffu, mbar_wait_relaxed(b0, p0, s_abort, g_status))) return false;
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    const bool t0 = d0 || mbar_test_relaxed(b0, p0);
-    const bool t1 = d1 || mbar_test_relaxed(b1, p1);
-    const bool t2 = d2 || mbar_test_relaxed(b2, p2);
-    d0 = t0; d1 = t1; d2 = t2;
-    if (__all_sync(0xffffffffu, d0 && d1 && d2)) return true;
+    const bool t1 = mbar_test_relaxed(b1, p1);
+    const bool t2 = mbar_test_relaxed(b2, p2);
+    if (__all_sync(0xffffffffu, t1 && t2)) return true;
     if (it > 1024 && *s_abort) return false;
   }
   *s_abort = 1;
@@ -125,13 +125,7 @@ __device__ __forceinline__ bool mbar_wait_all3(uint64_t* b0, uint32_t p0, uint64
 
 // The same for one barrier.
 __device__ __forceinline__ bool mbar_wait_all1(uint64_t* b0, uint32_t p0, volatile int* s_abort, int* g_status) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (__all_sync(0xffffffffu, mbar_test_relaxed(b0, p0))) return true;
-    if (it > 1024 && *s_abort) return false;
-  }
-  *s_abort = 1;
-  if (g_status) atomicExch(g_status, 10);
-  return false;
+  return __all_sync(0xffffffffu, mbar_wait_relaxed(b0, p0, s_abort, g_status));
 }
 
 // One lane of a fully active warp (the same lane every time for the same mask).
@@ -336,6 +330,13 @@ __device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
 __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
   f32x2 r;
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+  return r;
+}
+
+// max of three in one instruction
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
 
