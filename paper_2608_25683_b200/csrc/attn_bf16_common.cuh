@@ -35,6 +35,25 @@ __device__ __forceinline__ void load_kv_tile(uint8_t* dst, const CUtensorMap* ma
   }
 }
 
+// The same from host-resolved coordinates (TileLoad): no metadata load between the ring wait and
+// the TMA instructions.
+__device__ __forceinline__ void load_kv_tile_at(uint8_t* dst, const CUtensorMap* maps, uint64_t* bar, const TileLoad& tl,
+                                                int64_t head_row0) {
+  using namespace sm100;
+  const int rows_per_box = tl.bs >= 128 ? 128 : tl.bs;
+  const CUtensorMap* m = maps + map_index(tl.bs);
+  mbar_expect_tx(bar, uint32_t(tl.rows_loaded) * 256u);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if (i < tl.n_pages) {
+      uint8_t* d = dst + i * rows_per_box * 128;
+      const int row = int(head_row0 + tl.row[i]);
+      tma_load_2d(d, m, bar, 0, row);
+      tma_load_2d(d + kHalfBytes, m, bar, 64, row);
+    }
+  }
+}
+
 // One 128 x 128 row-tile of a [rows, Hq*128] tensor (Q, dO): head h, first row `row`.
 __device__ __forceinline__ void load_row_tile(uint8_t* dst, const CUtensorMap* m, uint64_t* bar, int h, int row) {
   sm100::tma_load_2d(dst, m, bar, h * 128, row);

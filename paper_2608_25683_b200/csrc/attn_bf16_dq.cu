@@ -41,7 +41,7 @@ struct Maps {
 };
 struct Params {
   const int32_t* blob;
-  int32_t off_qt, off_kvt, off_path_tiles, off_path_nvalid, off_page_slot;
+  int32_t off_qt, off_kvt, off_path_tiles, off_path_nvalid, off_path_loads, off_page_slot;
   int32_t Hq, G, T_q;
   int64_t cap;
   float scale, scale_log2;
@@ -71,7 +71,6 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int item = blockIdx.x / p.Hq, h = blockIdx.x % p.Hq, hk = h / p.G;
   const QTile qt = reinterpret_cast<const QTile*>(p.blob + p.off_qt)[item];
-  const int32_t* path_tiles = p.blob + p.off_path_tiles + qt.pt_begin;
   const int32_t* path_nvalid = p.blob + p.off_path_nvalid + qt.pt_begin;
   const int n_tiles = qt.n_kv_tiles;
 
@@ -100,16 +99,19 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       load_row_tile(sdO, &maps.d_o, &bar.qdo_full, h, qt.q_row0);
     }
     if (lane == 0) {
-      const KvTile* kvt = reinterpret_cast<const KvTile*>(p.blob + p.off_kvt);
-      const int32_t* page_slot = p.blob + p.off_page_slot;
+      // TMA coordinates of the item's KV tiles, resolved by the plan builder; the entry of tile j+1 is
+      // fetched while the ring waits of tile j run
+      const TileLoad* loads = reinterpret_cast<const TileLoad*>(p.blob + p.off_path_loads) + qt.pt_begin;
       const int64_t head_row0 = int64_t(hk) * p.cap;
+      TileLoad cur = loads[0];
       for (int j = 0; j < n_tiles; ++j) {
-        const KvTile kt = kvt[path_tiles[j]];
+        const TileLoad nxt = loads[j + 1 < n_tiles ? j + 1 : j];
         const int ks = j % KS, vs = j % VS;
-        if (j >= KS && !mbar_wait(&bar.k_empty[ks], ((j / KS) + 1) & 1, abortp, p.status)) break;
-        load_kv_tile(sK + ks * kTileBytes, maps.kv.k, &bar.k_full[ks], kt, page_slot, head_row0);
-        if (j >= VS && !mbar_wait(&bar.v_empty[vs], ((j / VS) + 1) & 1, abortp, p.status)) break;
-        load_kv_tile(sV + vs * kTileBytes, maps.kv.v, &bar.v_full[vs], kt, page_slot, head_row0);
+        if (j >= KS && !mbar_wait_sleepy(&bar.k_empty[ks], ((j / KS) + 1) & 1, abortp, p.status)) break;
+        load_kv_tile_at(sK + ks * kTileBytes, maps.kv.k, &bar.k_full[ks], cur, head_row0);
+        if (j >= VS && !mbar_wait_sleepy(&bar.v_empty[vs], ((j / VS) + 1) & 1, abortp, p.status)) break;
+        load_kv_tile_at(sV + vs * kTileBytes, maps.kv.v, &bar.v_full[vs], cur, head_row0);
+        cur = nxt;
       }
     }
   } else if (warp == 9) {
@@ -300,7 +302,7 @@ psrl_status_t dq_bf16(const AttnArgs& a) {
   Params p{};
   p.blob = P.dev;
   p.off_qt = H.off_qt; p.off_kvt = H.off_kvt; p.off_path_tiles = H.off_path_tiles;
-  p.off_path_nvalid = H.off_path_nvalid; p.off_page_slot = H.off_page_slot;
+  p.off_path_nvalid = H.off_path_nvalid; p.off_path_loads = H.off_path_loads; p.off_page_slot = H.off_page_slot;
   p.Hq = P.Hq; p.G = P.Hq / P.Hkv; p.T_q = P.T_q;
   p.cap = cap; p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
   p.lse = a.lse_in; p.delta = a.delta; p.d_q = static_cast<__nv_bfloat16*>(a.d_q); p.status = a.status;

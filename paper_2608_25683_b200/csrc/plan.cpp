@@ -488,6 +488,15 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
     P.path_nvalid.resize(P.path_tiles.size());
     for (size_t i = 0; i < P.path_tiles.size(); ++i) P.path_nvalid[i] = P.kv_tiles[P.path_tiles[i]].n_valid;
     H.off_path_nvalid = append_array(B, P.path_nvalid);
+    P.path_loads.resize(P.path_tiles.size());
+    for (size_t i = 0; i < P.path_tiles.size(); ++i) {
+      const KvTile& kt = P.kv_tiles[P.path_tiles[i]];
+      TileLoad& tl = P.path_loads[i];
+      tl = TileLoad{};
+      tl.n_pages = kt.n_pages; tl.bs = kt.bs; tl.rows_loaded = kt.rows_loaded;
+      for (int32_t pg = 0; pg < kt.n_pages && pg < 8; ++pg) tl.row[pg] = P.page_slot[kt.first_page + pg] + kt.row_off;
+    }
+    H.off_path_loads = append_array(B, P.path_loads);
     H.n_kvi = static_cast<int32_t>(P.kv_items.size());
     H.off_split = append_array(B, P.kv_splits);
     H.n_split = static_cast<int32_t>(P.kv_splits.size());

@@ -26,6 +26,14 @@ struct KvTile {
   int32_t pad0, pad1, pad2;
 };
 
+// TMA coordinates of one entry of a KV-tile list, resolved on the host so that the producer
+// thread of the forward / dQ kernels needs one load per tile instead of a chain of three
+// (list entry -> tile record -> page slots): first pool row (slot) of each page of the tile.
+struct TileLoad {
+  int32_t n_pages, bs, rows_loaded, pad;
+  int32_t row[8];   // a tile spans at most 8 pages (page size >= 16 slots)
+};
+
 // One work item of the forward and dQ kernels: up to 128 consecutive query rows
 // and a list of KV tiles they attend to.
 //  * own item: rows of one HAS_Q segment; the list holds the tiles of its
@@ -84,12 +92,13 @@ struct DeviceHeader {
   int32_t off_qrow_seg;  // [T_q] segment of every query row
   int32_t off_kvt, off_qt, off_kvi, off_path_off, off_path_tiles;
   int32_t off_path_nvalid;  // valid keys of every entry of path_tiles
+  int32_t off_path_loads;   // TileLoad of every entry of path_tiles
   int32_t n_kvi;
   int32_t n_split, off_split, n_slabs;
   // merge lists of the rows that are assembled from partial results: row i of the list is
   // query row merge_row[i]; its parts are merge_parts[merge_off[i] .. merge_off[i+1]) (partial-row ids)
   int32_t n_part_rows, n_merge_rows, off_merge_row, off_merge_off, off_merge_parts;
-  int32_t reserved[2];
+  int32_t reserved[1];
 };
 
 struct Plan {
@@ -113,6 +122,7 @@ struct Plan {
   std::vector<uint8_t> seg_cascaded;  // 1: the segment's KV tiles are handled by packed items
   int32_t n_part_rows = 0;
   std::vector<int32_t> merge_row, merge_off, merge_parts;
+  std::vector<TileLoad> path_loads;
   std::vector<int32_t> seg_first_kvt, seg_n_kvt, seg_desc_q_begin, seg_desc_q_end, path_off, path_tiles, path_nvalid, qrow_seg;
   // device blob
   std::vector<int32_t> blob;

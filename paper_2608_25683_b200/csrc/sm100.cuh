@@ -61,6 +61,21 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
+// Bounded wait of a TMA producer thread on a ring stage.  The producer is usually ahead and
+// spends most of its time here; it sleeps between polls so that it takes no issue slots from the
+// softmax warps of its SM sub-partition.
+__device__ __forceinline__ bool mbar_wait_sleepy(uint64_t* bar, uint32_t parity, volatile int* s_abort,
+                                                 int* g_status) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    __nanosleep(128);
+    if (it > 64 && *s_abort) return false;
+  }
+  *s_abort = 1;
+  if (g_status) atomicExch(g_status, 10);
+  return false;
+}
+
 // The same bounded wait for the MMA-issuing thread.  An acquire-ordered
 // mbarrier wait stalls that thread for ~100 cycles while MMAs are in flight
 // (measured), which starves the tensor cores; the relaxed form does not.  The
