@@ -143,25 +143,45 @@ def oracle_leg(w, n_keep, seed, steps=1, warmup=0):
     from oracle import oracle_attn, oracle_plan
     from paper_2608_25683_b200.workloads import make_inputs
 
-    sw = sub_workload(w, n_keep)
-    plan = oracle_plan(sw.parent, sw.seg_len, sw.group_block_size, sw.seg_flags, None)
+    # Bound the sample: the oracle materialises every sample unshared, so its cost follows the flat pair
+    # count.  Fewer samples first; if one sample alone is too large (c5), an evenly spaced subset of the
+    # query rows (exact for those rows: the other dO rows are taken as zero).
+    G = w.n_q_heads // w.n_kv_heads
+    budget = 1.5e12   # fp64 FLOP of flat work per pass: 10-30 s on the host cores of this pool
+    while True:
+        sw = sub_workload(w, n_keep)
+        plan = oracle_plan(sw.parent, sw.seg_len, sw.group_block_size, sw.seg_flags, None)
+        flat_flops = dedup_flops(sw.head_dim, G, plan["flat_pairs"])
+        if flat_flops <= budget or n_keep == 1:
+            break
+        n_keep -= 1
     q, k, v, d_o = make_inputs(plan["T_q"], plan["pool_slots"], plan["tok_slot"], sw.n_q_heads, sw.n_kv_heads,
                                sw.head_dim, sw.dtype, seed, device="cpu")
     f = lambda t: t.float().numpy()
     q, k, v, d_o = f(q), f(k), f(v), f(d_o)
-    G = sw.n_q_heads // sw.n_kv_heads
-    flops = dedup_flops(sw.head_dim, G, plan["tree_pairs"])
+    q_rows, rows_note = None, ""
+    if flat_flops > budget:
+        stride = int(np.ceil(flat_flops / budget))
+        q_rows = np.arange(0, plan["T_q"], stride, dtype=np.int64)
+        q, d_o = q[q_rows], d_o[q_rows]
+        seg_of = np.repeat(np.arange(plan["n_seg"]), np.where(plan["seg_q_off"] >= 0, plan["seg_len"], 0))
+        pos = q_rows - plan["seg_q_off"][seg_of[q_rows]]
+        pairs = int(np.sum(plan["seg_anc_tokens"][seg_of[q_rows]].astype(np.int64) + pos + 1))
+        flops = dedup_flops(sw.head_dim, G, pairs)
+        rows_note = f", every {stride}th query row ({len(q_rows)} rows)"
+    else:
+        flops = dedup_flops(sw.head_dim, G, plan["tree_pairs"])
     times = []
     for i in range(warmup + steps):
         t0 = time.perf_counter()
-        oracle_attn(plan, q, k, v, d_o, sw.softmax_scale, kv_heads=[0])
+        oracle_attn(plan, q, k, v, d_o, sw.softmax_scale, kv_heads=[0], q_rows=q_rows)
         if i >= warmup:
             times.append(time.perf_counter() - t0)
     t = float(np.mean(times))
     cores = len(os.sched_getaffinity(0))
     return dict(value=flops / t / 1e12, unit=UNIT, cores=cores, kind="oracle",
                 sample=f"KV head 0 ({G} query heads) of the first {plan['n_samples']} samples of {w.name} "
-                       f"(seed {w.seed}): {plan['T']} tree tokens, {plan['flat_tokens']} unshared tokens, "
+                       f"(seed {w.seed}){rows_note}: {plan['T']} tree tokens, {plan['flat_tokens']} unshared tokens, "
                        f"{flops:.3e} dedup FLOP, {t:.2f} s per pass (numpy fp64, torch threads "
                        f"{torch.get_num_threads()})"), t
 
