@@ -72,6 +72,12 @@ typedef struct {
   psrl_dtype_t dtype;
   const int32_t* free_extents;     /* [2 * n_free] (start_slot, n_slots), multiples of 16; NULL = bump from 0 */
   int32_t n_free;
+  /* Optional [n_segments] (input order) or NULL: where a segment's K/V already lives.  A value >= 0
+   * (a multiple of 16) pins the segment: its pages are the consecutive runs of block-size slots starting
+   * there and take nothing from the free extents; -1 allocates as usual.  This is how a prefix cached
+   * by an earlier micro-batch is reused in place (paper Sec. 4.1 inter-batch / self-sequence sharing,
+   * Sec. 5.2): the cache manager (psrl_cache.h) hands out these bases. */
+  const int32_t* seg_slot_base;
 } psrl_tree_desc_t;
 
 typedef struct psrl_plan psrl_plan_t;

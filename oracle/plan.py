@@ -46,7 +46,7 @@ def _i32(x):
     return np.asarray(x, dtype=np.int32)
 
 
-def oracle_plan(parent, seg_len, group_block_size, seg_flags=None, free_extents=None):
+def oracle_plan(parent, seg_len, group_block_size, seg_flags=None, free_extents=None, seg_slot_base=None):
     """Build the canonical plan.
 
     parent[s]            -1 for a root, else an input index < s
@@ -57,6 +57,11 @@ def oracle_plan(parent, seg_len, group_block_size, seg_flags=None, free_extents=
                          SAMPLE_END on leaves
     free_extents         None = one unbounded extent starting at slot 0, else a
                          list of (start_slot, n_slots), all multiples of 16
+    seg_slot_base[s]     None, or per segment: >= 0 (a multiple of 16) pins the
+                         segment's pages to consecutive runs of block-size slots
+                         from that slot on (K/V cached by an earlier micro-batch,
+                         Sec. 4.1 / 5.2) and takes nothing from the free extents;
+                         -1 allocates as usual
 
     Returns a dict of python ints and numpy int32 arrays (int64 where noted).
     """
@@ -101,6 +106,14 @@ def oracle_plan(parent, seg_len, group_block_size, seg_flags=None, free_extents=
         for a, c in free_extents:
             if a < 0 or c < 0 or a % 16 or c % 16:
                 raise PlanError("INVALID_ARG", "free extent not a multiple of 16")
+
+    if seg_slot_base is not None:
+        seg_slot_base = [int(b) for b in seg_slot_base]
+        if len(seg_slot_base) != n:
+            raise PlanError("INVALID_ARG", "seg_slot_base length")
+        for b in seg_slot_base:
+            if b < -1 or (b >= 0 and b % 16):
+                raise PlanError("INVALID_ARG", "seg_slot_base not -1 or a multiple of 16")
 
     # -- step 2: canonical order = DFS preorder --------------------------------
     input_of_canon = []
@@ -178,9 +191,12 @@ def oracle_plan(parent, seg_len, group_block_size, seg_flags=None, free_extents=
         npg = -(-c_len[c] // bs)
         c_first_page[c] = len(page_seg)
         c_n_pages[c] = npg
+        pinned = -1 if seg_slot_base is None else seg_slot_base[input_of_canon[c]]
         for i in range(npg):
             valid = bs if i < npg - 1 else c_len[c] - (npg - 1) * bs
-            if extents is None:
+            if pinned >= 0:
+                slot = pinned + i * bs
+            elif extents is None:
                 slot = bump
                 bump += bs
             else:

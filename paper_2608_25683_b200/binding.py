@@ -38,6 +38,7 @@ class TreeDesc(C.Structure):
         ("n_segments", C.c_int32), ("parent", _I32P), ("seg_len", _I32P), ("seg_flags", C.POINTER(C.c_uint8)),
         ("group_block_size", _I32P), ("n_groups", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
         ("head_dim", C.c_int32), ("dtype", C.c_int), ("free_extents", _I32P), ("n_free", C.c_int32),
+        ("seg_slot_base", _I32P),
     ]
 
 
@@ -137,7 +138,7 @@ class Plan:
 
     def __init__(self, parent: Sequence[int], seg_len: Sequence[int], group_block_size: Sequence[int],
                  n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: str,
-                 seg_flags: Optional[Sequence[int]] = None, free_extents=None):
+                 seg_flags: Optional[Sequence[int]] = None, free_extents=None, seg_slot_base=None):
         self._h = C.c_void_p()
         self._dev = None
         self._ws = {}
@@ -160,6 +161,12 @@ class Plan:
             fe = _i32(np.asarray(free_extents, dtype=np.int64).reshape(-1))
             d.free_extents = fe.ctypes.data_as(_I32P)
             d.n_free = len(fe) // 2
+        sb = None
+        if seg_slot_base is not None:
+            sb = _i32(seg_slot_base)
+            if len(sb) != len(p):
+                raise ValueError("seg_slot_base needs one entry per segment")
+            d.seg_slot_base = sb.ctypes.data_as(_I32P)
         _check(L.psrl_plan_build(C.byref(d), C.byref(self._h)), "psrl_plan_build")
         self.n_q_heads, self.n_kv_heads, self.head_dim, self.dtype = int(n_q_heads), int(n_kv_heads), int(head_dim), dtype
         v = PlanView()

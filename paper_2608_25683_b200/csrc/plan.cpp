@@ -99,6 +99,12 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
       extents.push_back({a, c});
     }
 
+    if (desc.seg_slot_base)
+      for (int32_t s = 0; s < n; ++s) {
+        const int64_t b = desc.seg_slot_base[s];
+        if (b < -1 || (b >= 0 && b % 16)) return PSRL_ERR_INVALID_ARG;
+      }
+
     // ---- canonical order: preorder walk with sibling links ----
     P.input_of_canon.reserve(n);
     P.canon_of_input.assign(n, -1);
@@ -177,9 +183,12 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
       const int32_t npg = (len + bs - 1) / bs;
       P.seg_first_page[c] = static_cast<int32_t>(P.page_seg.size());
       P.seg_n_pages[c] = npg;
+      const int64_t pinned = desc.seg_slot_base ? desc.seg_slot_base[P.input_of_canon[c]] : -1;
       for (int32_t i = 0; i < npg; ++i) {
         int64_t slot = -1;
-        if (bump) {
+        if (pinned >= 0) {
+          slot = pinned + int64_t(i) * bs;
+        } else if (bump) {
           slot = bump_at;
           bump_at += bs;
         } else {

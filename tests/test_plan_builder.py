@@ -134,3 +134,44 @@ def test_flatten_forest(lib):
     assert first.sum() == V["T"]
     flat = lib.Plan(parent, seg_len, gbs, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype)
     assert flat.view["tree_pairs"] == V["flat_pairs"] == flat.view["flat_pairs"]
+
+
+def test_pinned_segments_bit_exact(lib):
+    """Segments whose K/V already lives in the pool (cached by an earlier micro-batch) are pinned
+    to their slots; everything else is allocated around them exactly as the oracle does."""
+    rng = np.random.default_rng(77)
+    for it in range(25):
+        n_roots = 1 + it % 2
+        parent, seg_len, gbs, flags = random_forest(rng, int(rng.integers(n_roots + 1, 12)), 300, n_roots,
+                                                    cached_roots=(it % 3 == 0))
+        # pin a random subset at non-overlapping bases far above the bump region
+        base, pinned, at = [], rng.random(len(parent)) < 0.4, 1 << 16
+        root_of = []
+        for s, p in enumerate(parent):
+            root_of.append(len([q for q in parent[:s + 1] if q == -1]) - 1 if p == -1 else root_of[p])
+        for s in range(len(parent)):
+            if pinned[s]:
+                bs = gbs[root_of[s]]
+                base.append(at)
+                at += -(-seg_len[s] // bs) * bs + 16 * int(rng.integers(0, 4))
+            else:
+                base.append(-1)
+        want = oracle_plan(parent, seg_len, gbs, flags, None, base)
+        got = lib.Plan(parent, seg_len, gbs, 4, 2, 128, "bf16", seg_flags=flags, seg_slot_base=base).view
+        for name in PLAN_ARRAYS:
+            assert np.array_equal(got[name], want[name]), name
+        for name in PLAN_SCALARS:
+            assert int(got[name]) == int(want[name]), name
+        # pinned pages sit where they were put
+        for s in range(len(parent)):
+            if base[s] >= 0:
+                c = int(want["canon_of_input"][s])
+                p0 = int(want["seg_first_page"][c])
+                assert int(want["page_slot"][p0]) == base[s]
+    # a base that is not a multiple of 16 is rejected by both
+    with pytest.raises(PlanError) as e1:
+        oracle_plan([-1, 0], [20, 5], [16], None, None, [8, -1])
+    assert e1.value.code == "INVALID_ARG"
+    with pytest.raises(lib.PsrlError) as e2:
+        lib.Plan([-1, 0], [20, 5], [16], 4, 2, 128, "bf16", seg_slot_base=[8, -1])
+    assert e2.value.name == "PSRL_ERR_INVALID_ARG"
