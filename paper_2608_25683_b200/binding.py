@@ -28,6 +28,8 @@ EXPORTS = [
     "psrl_fwd_workspace_bytes", "psrl_bwd_workspace_bytes", "psrl_tree_attn_fwd", "psrl_tree_attn_bwd",
     "psrl_device_status", "psrl_last_cuda_error", "psrl_plan_destroy", "psrl_status_string",
     "psrl_profile_bwd_phases", "psrl_tree_attn_bwd_static", "psrl_launch_count", "psrl_plan_schedule",
+    "psrl_cache_create", "psrl_cache_begin", "psrl_cache_end", "psrl_cache_stats", "psrl_cache_refcounts",
+    "psrl_cache_destroy",
 ]
 
 _I32P = C.POINTER(C.c_int32)
@@ -40,6 +42,29 @@ class TreeDesc(C.Structure):
         ("head_dim", C.c_int32), ("dtype", C.c_int), ("free_extents", _I32P), ("n_free", C.c_int32),
         ("seg_slot_base", _I32P),
     ]
+
+
+class CacheDesc(C.Structure):
+    _fields_ = [
+        ("n_segments", C.c_int32), ("parent", _I32P), ("seg_len", _I32P), ("seg_flags", C.POINTER(C.c_uint8)),
+        ("group_block_size", _I32P), ("n_groups", C.c_int32), ("n_microbatches", C.c_int32), ("mb_of_seg", _I32P),
+        ("capacity_slots", C.c_int64),
+    ]
+
+
+class CacheStep(C.Structure):
+    _fields_ = [
+        ("n_segments", C.c_int32), ("seg_id", _I32P), ("parent", _I32P), ("seg_len", _I32P),
+        ("seg_flags", C.POINTER(C.c_uint8)), ("group_block_size", _I32P), ("n_groups", C.c_int32),
+        ("seg_slot_base", _I32P), ("n_new", C.c_int32), ("n_reload", C.c_int32), ("n_evict", C.c_int32),
+        ("new_seg", _I32P), ("reload_seg", _I32P), ("evict_seg", _I32P), ("evict_base", _I32P),
+        ("live_slots", C.c_int64), ("pool_slots", C.c_int64),
+    ]
+
+
+class CacheStats(C.Structure):
+    _fields_ = [("peak_slots", C.c_int64), ("evicted_slots", C.c_int64), ("reloaded_slots", C.c_int64),
+                ("pool_high_water", C.c_int64), ("total_slots", C.c_int64)]
 
 
 _VIEW_SCALARS32 = ["n_seg", "n_groups", "n_pages", "n_samples", "max_depth", "T", "T_q", "pool_slots"]
@@ -110,6 +135,18 @@ def lib() -> C.CDLL:
     L.psrl_profile_bwd_phases.restype = C.c_int
     L.psrl_plan_schedule.argtypes = [C.c_void_p, C.POINTER(_I32P), C.POINTER(C.c_size_t)]
     L.psrl_plan_schedule.restype = C.c_int
+    L.psrl_cache_create.argtypes = [C.POINTER(CacheDesc), C.POINTER(C.c_void_p)]
+    L.psrl_cache_create.restype = C.c_int
+    L.psrl_cache_begin.argtypes = [C.c_void_p, C.c_int32, C.POINTER(CacheStep)]
+    L.psrl_cache_begin.restype = C.c_int
+    L.psrl_cache_end.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(_I32P), C.POINTER(C.c_int64)]
+    L.psrl_cache_end.restype = C.c_int
+    L.psrl_cache_stats.argtypes = [C.c_void_p, C.POINTER(CacheStats)]
+    L.psrl_cache_stats.restype = C.c_int
+    L.psrl_cache_refcounts.argtypes = [C.c_void_p, C.POINTER(_I32P)]
+    L.psrl_cache_refcounts.restype = C.c_int
+    L.psrl_cache_destroy.argtypes = [C.c_void_p]
+    L.psrl_cache_destroy.restype = None
     L.psrl_launch_count.argtypes = [C.c_void_p, C.c_int]
     L.psrl_launch_count.restype = C.c_int
     L.psrl_last_cuda_error.restype = C.c_char_p
@@ -327,6 +364,63 @@ def psrl_profile_bwd_phases(mask: int) -> int:
     """Profiling aid: choose which backward kernels the next calls launch
     (bit 0 delta pre-pass, bit 1 dQ, bit 2 dK/dV); returns the previous mask."""
     return int(lib().psrl_profile_bwd_phases(int(mask)))
+
+
+class Cache:
+    """Owner of a psrl_cache_t (Dynamic Block Caching over an ordered list of micro-batches).
+    begin(m) returns the micro-batch's tree as plain lists, ready for Plan(..., seg_slot_base=...)."""
+
+    def __init__(self, parent, seg_len, group_block_size, mb_of_seg, n_microbatches: int, seg_flags=None,
+                 capacity_slots: int = 0):
+        self._h = C.c_void_p()
+        p, l, g, mb = _i32(parent), _i32(seg_len), _i32(group_block_size), _i32(mb_of_seg)
+        d = CacheDesc()
+        d.n_segments = len(p)
+        d.parent, d.seg_len = p.ctypes.data_as(_I32P), l.ctypes.data_as(_I32P)
+        fl = None
+        if seg_flags is not None:
+            fl = np.ascontiguousarray(np.asarray(seg_flags, dtype=np.uint8))
+            d.seg_flags = fl.ctypes.data_as(C.POINTER(C.c_uint8))
+        d.group_block_size, d.n_groups = g.ctypes.data_as(_I32P), len(g)
+        d.n_microbatches = int(n_microbatches)
+        if len(mb) != len(p) or len(l) != len(p):
+            raise ValueError("parent, seg_len and mb_of_seg need one entry per segment")
+        d.mb_of_seg = mb.ctypes.data_as(_I32P)
+        d.capacity_slots = int(capacity_slots)
+        self.n_segments = len(p)
+        _check(lib().psrl_cache_create(C.byref(d), C.byref(self._h)), "psrl_cache_create")
+
+    def begin(self, m: int) -> dict:
+        st = CacheStep()
+        _check(lib().psrl_cache_begin(self._h, int(m), C.byref(st)), "psrl_cache_begin")
+        arr = lambda ptr, k: [int(ptr[i]) for i in range(k)]
+        k = st.n_segments
+        return dict(seg_id=arr(st.seg_id, k), parent=arr(st.parent, k), seg_len=arr(st.seg_len, k),
+                    seg_flags=arr(st.seg_flags, k), group_block_size=arr(st.group_block_size, st.n_groups),
+                    seg_slot_base=arr(st.seg_slot_base, k), new=arr(st.new_seg, st.n_new),
+                    reload=arr(st.reload_seg, st.n_reload),
+                    evict=list(zip(arr(st.evict_seg, st.n_evict), arr(st.evict_base, st.n_evict))),
+                    live_slots=int(st.live_slots), pool_slots=int(st.pool_slots))
+
+    def end(self, m: int) -> dict:
+        nf, ptr, live = C.c_int32(), _I32P(), C.c_int64()
+        _check(lib().psrl_cache_end(self._h, int(m), C.byref(nf), C.byref(ptr), C.byref(live)), "psrl_cache_end")
+        return dict(freed=[int(ptr[i]) for i in range(nf.value)], live_slots=int(live.value))
+
+    def stats(self) -> dict:
+        s = CacheStats()
+        _check(lib().psrl_cache_stats(self._h, C.byref(s)), "psrl_cache_stats")
+        return {n: int(getattr(s, n)) for n, _ in CacheStats._fields_}
+
+    def refcounts(self):
+        ptr = _I32P()
+        _check(lib().psrl_cache_refcounts(self._h, C.byref(ptr)), "psrl_cache_refcounts")
+        return [int(ptr[i]) for i in range(self.n_segments)]
+
+    def __del__(self):
+        if getattr(self, "_h", None) and self._h.value:
+            lib().psrl_cache_destroy(self._h)
+            self._h = C.c_void_p()
 
 
 def psrl_launch_count(plan: Plan, backward: bool) -> int:

@@ -91,12 +91,12 @@ def test_errors_match_oracle(lib):
 
 
 def test_library_exports_every_declared_symbol(lib):
-    hdr = open(os.path.join(ROOT, "include", "psrl.h")).read()
+    hdr = open(os.path.join(ROOT, "include", "psrl.h")).read() + open(os.path.join(ROOT, "include", "psrl_cache.h")).read()
     declared = set(re.findall(r"\b(psrl_[a-z_0-9]+)\s*\(", hdr))
     assert declared, "no declarations found"
     L = lib.lib()
     for name in declared:
-        assert hasattr(L, name), f"{name} declared in include/psrl.h but not exported"
+        assert hasattr(L, name), f"{name} declared in include/*.h but not exported"
     assert set(lib.EXPORTS) <= declared
     assert L.psrl_status_string(0) == b"PSRL_OK"
     assert L.psrl_status_string(10) == b"PSRL_ERR_TIMEOUT"
