@@ -337,6 +337,64 @@ def flat_runner(lib, r, device, head_slice=None):
     return Runner(lib, fw, 0, device, data=(q, k, v, d_o))
 
 
+def microbatch_leg(lib, w, device, flops, seed, iters):
+    """The same forest run as an ordered list of micro-batches (Sec. 4.1): every root is computed with its
+    first child, every further child of a root in a micro-batch of its own (deeper levels follow their
+    parent's micro-batch or later, breadth first).  Cached prefixes are read in place; the Dynamic Block
+    Caching manager (Sec. 5.2) assigns extents and releases blocks after their last use.  Timed: all
+    forward + backward calls of the micro-batches; plans are built and uploaded beforehand."""
+    import torch
+
+    n = len(w.parent)
+    children = [[] for _ in range(n)]
+    for s, p in enumerate(w.parent):
+        if p >= 0:
+            children[p].append(s)
+    mb = [0] * n
+    for s in range(n):                      # parents come before children
+        for i, c in enumerate(children[s]):
+            mb[c] = mb[s] + i
+    M = max(mb) + 1
+    cache = lib.Cache(w.parent, w.seg_len, w.group_block_size, mb, M, seg_flags=w.seg_flags)
+    arena = cache.stats()["total_slots"]
+    Hq, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
+    dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    g = torch.Generator(device=device).manual_seed(seed)
+    K = torch.randn(Hkv, arena, d, generator=g, device=device, dtype=torch.float32).to(dt)
+    V = torch.randn(Hkv, arena, d, generator=g, device=device, dtype=torch.float32).to(dt)
+    dK, dV = torch.zeros_like(K), torch.zeros_like(V)
+    steps, trace, t_plan = [], [], 0.0
+    for m in range(M):
+        st = cache.begin(m)
+        t0 = time.perf_counter()
+        plan = lib.Plan(st["parent"], st["seg_len"], st["group_block_size"], Hq, Hkv, d, w.dtype,
+                        seg_flags=st["seg_flags"], seg_slot_base=st["seg_slot_base"]).upload(device)
+        t_plan += time.perf_counter() - t0
+        T_q = plan.view["T_q"]
+        q = torch.randn(T_q, Hq, d, generator=g, device=device, dtype=torch.float32).to(dt)
+        d_o = torch.randn(T_q, Hq, d, generator=g, device=device, dtype=torch.float32).to(dt)
+        o, dq = torch.empty_like(q), torch.empty_like(q)
+        lse = torch.empty((Hq, T_q), dtype=torch.float32, device=device)
+        steps.append((plan, q, d_o, o, lse, dq))
+        after = cache.end(m)["live_slots"]
+        trace.append([st["live_slots"], after])
+
+    def run():
+        for plan, q, d_o, o, lse, dq in steps:
+            lib.psrl_tree_attn_fwd(plan, q, K, V, w.softmax_scale, o=o, lse=lse)
+            lib.psrl_tree_attn_bwd(plan, q, K, V, o, lse, d_o, w.softmax_scale, d_q=dq, dk_pool=dK, dv_pool=dV)
+
+    ms = time_region(run, iters, 2)
+    for plan, *_ in steps:
+        assert lib.psrl_device_status(plan, "bwd") == 0
+    st = cache.stats()
+    return {"n_microbatches": M, "ms_all_microbatches": round(ms, 4), "dedup_tflops": round(flops / (ms * 1e-3) / 1e12, 2),
+            "plan_build_upload_ms": round(t_plan * 1e3, 2), "peak_kv_slots": st["peak_slots"],
+            "kv_slots_without_caching_policy": st["total_slots"],
+            "peak_reduction": round(1 - st["peak_slots"] / st["total_slots"], 4),
+            "live_slots_during_after": trace if M <= 64 else trace[:64]}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -349,6 +407,8 @@ def main():
     ap.add_argument("--ref-samples", type=int, default=2, help="samples per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unshared", action="store_true")
+    ap.add_argument("--microbatch", action="store_true",
+                    help="also run the group as one micro-batch per branch with the Dynamic Block Caching manager")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -500,6 +560,10 @@ def main():
         except Exception as ex:  # e.g. out of memory on the flattened tensors
             unshared = {"error": str(ex)[:200]}
 
+    micro = None
+    if args.microbatch and world == 1:
+        micro = microbatch_leg(lib, w, device, flops, args.seed + 7, max(3, min(args.steps, 10)))
+
     cpu = None
     if not args.no_cpu_baseline:
         cpu, _ = oracle_leg(w, args.cpu_samples, args.seed + 1)
@@ -511,7 +575,7 @@ def main():
                     "per-step working set exceeds the 126 MB L2 (inputs larger than L2); no explicit flush" if flush is None
                     else "working set fits in the L2: a 252 MB buffer is overwritten before every timed step "
                          "(each step timed on its own, flush outside the timed part)")), clocks=clocks.summary(), e2e=e2e, gpu_launches=(lib.psrl_launch_count(r.plan, False) + lib.psrl_launch_count(r.plan, True)) * args.steps,
-                roofline=roofline, cpu_baseline=cpu, unshared=unshared,
+                roofline=roofline, cpu_baseline=cpu, unshared=unshared, microbatch=micro,
                 frac_of_bf16_peak={"burst": round(value / world / pk["bf16_tflops"], 4),
                                    "sustained": round(value / world / pk["bf16_tflops_sustained"], 4)})
     print(json.dumps(line), flush=True)
