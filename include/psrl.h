@@ -34,7 +34,9 @@ typedef enum {
   PSRL_OK = 0,
   PSRL_ERR_INVALID_ARG = 1,    /* null / misaligned pointer, bad count, bad flag bits */
   PSRL_ERR_BAD_TREE = 2,       /* parent >= own index, length < 1, leaf that ends no sample */
-  PSRL_ERR_BAD_BLOCK_SIZE = 3, /* block size not a power of two in [16, 256] */
+  PSRL_ERR_BAD_BLOCK_SIZE = 3, /* block size not a power of two in [16, 256], or 0 =
+                                      adaptive (Sec. 5.1): one extent per segment sized to its span at 16-slot
+                                      granularity (bf16 path only) */
   PSRL_ERR_SHAPE = 4,          /* head counts do not divide, pool smaller than the plan needs */
   PSRL_ERR_UNSUPPORTED = 5,    /* dtype x head_dim outside {f32 x {64,128}, bf16 x 128} */
   PSRL_ERR_POOL_FULL = 6,      /* no free extent fits a page */
@@ -65,7 +67,9 @@ typedef struct {
   const int32_t* parent;           /* [n_segments] -1 = root, else an index < own index */
   const int32_t* seg_len;          /* [n_segments] tokens, >= 1 */
   const uint8_t* seg_flags;        /* [n_segments] or NULL = HAS_Q everywhere, SAMPLE_END on leaves */
-  const int32_t* group_block_size; /* one per root, in input order; power of two in [16, 256] */
+  const int32_t* group_block_size; /* one per root, in input order; power of two in [16, 256], or 0 =
+                                      adaptive (Sec. 5.1): one extent per segment sized to its span at 16-slot
+                                      granularity (bf16 path only) */
   int32_t n_groups;                /* must equal the number of roots */
   int32_t n_q_heads, n_kv_heads;   /* n_q_heads % n_kv_heads == 0 */
   int32_t head_dim;                /* 64 or 128 (f32), 128 (bf16) */

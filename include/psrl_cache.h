@@ -39,7 +39,9 @@ typedef struct {
   const int32_t* parent;           /* [n_segments] -1 = root, else an index < own index */
   const int32_t* seg_len;          /* [n_segments] tokens, >= 1 */
   const uint8_t* seg_flags;        /* [n_segments] PSRL_SEG_SAMPLE_END bits, or NULL = leaves end samples */
-  const int32_t* group_block_size; /* one per root, in input order; power of two in [16, 256] */
+  const int32_t* group_block_size; /* one per root, in input order; power of two in [16, 256], or 0 =
+                                      adaptive (Sec. 5.1): one extent per segment sized to its span at 16-slot
+                                      granularity (bf16 path only) */
   int32_t n_groups;                /* must equal the number of roots */
   int32_t n_microbatches;          /* >= 1 */
   const int32_t* mb_of_seg;        /* [n_segments] micro-batch that computes the segment; a prefix is

@@ -61,7 +61,7 @@ class OracleCache:
         if len(group_block_size) != len(roots):
             raise CacheError("INVALID_ARG", "one block size per root")
         for b in group_block_size:
-            if b < 16 or b > 256 or (b & (b - 1)):
+            if b != 0 and (b < 16 or b > 256 or (b & (b - 1))):
                 raise CacheError("BAD_BLOCK_SIZE", str(b))
         if self.capacity < 0 or self.capacity % 16:
             raise CacheError("INVALID_ARG", "capacity")
@@ -72,7 +72,8 @@ class OracleCache:
             self.group[s] = roots.index(s) if self.parent[s] == -1 else self.group[self.parent[s]]
         self.gbs = [int(b) for b in group_block_size]
         self.bs = [self.gbs[self.group[s]] for s in range(n)]
-        self.extent = [-(-self.seg_len[s] // self.bs[s]) * self.bs[s] for s in range(n)]
+        # block size 0 = adaptive (Sec. 5.1): the span at 16-slot granularity
+        self.extent = [-(-self.seg_len[s] // (self.bs[s] or 16)) * (self.bs[s] or 16) for s in range(n)]
         if sample_end is None:
             self.sample_end = [not children[s] for s in range(n)]
         else:

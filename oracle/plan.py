@@ -52,7 +52,11 @@ def oracle_plan(parent, seg_len, group_block_size, seg_flags=None, free_extents=
     parent[s]            -1 for a root, else an input index < s
     seg_len[s]           tokens in segment s (>= 1)
     group_block_size[g]  page size of the g-th root (roots counted in input
-                         order); power of two in [16, 256]
+                         order); power of two in [16, 256], or 0 = adaptive
+                         (Sec. 5.1): every segment of the group gets ONE
+                         contiguous extent sized to its span at 16-slot
+                         granularity, recorded as pages of 128 slots followed
+                         by pages of 16 slots for the tail
     seg_flags[s]         bit 0 HAS_Q, bit 1 SAMPLE_END; None = HAS_Q everywhere,
                          SAMPLE_END on leaves
     free_extents         None = one unbounded extent starting at slot 0, else a
@@ -99,7 +103,7 @@ def oracle_plan(parent, seg_len, group_block_size, seg_flags=None, free_extents=
     if len(gbs) != len(roots):
         raise PlanError("INVALID_ARG", "one block size per root")
     for b in gbs:
-        if b < 16 or b > 256 or (b & (b - 1)):
+        if b != 0 and (b < 16 or b > 256 or (b & (b - 1))):
             raise PlanError("BAD_BLOCK_SIZE", str(b))
     if free_extents is not None:
         free_extents = [(int(a), int(c)) for a, c in free_extents]
@@ -186,35 +190,46 @@ def oracle_plan(parent, seg_len, group_block_size, seg_flags=None, free_extents=
     page_seg, page_bs, page_valid, page_pos, page_ref, page_slot = [], [], [], [], [], []
     extents = None if free_extents is None else [list(e) for e in free_extents]
     bump = 0
+    def take(size):
+        nonlocal bump
+        if extents is None:
+            slot = bump
+            bump += size
+            return slot
+        for e in extents:
+            if e[1] >= size:
+                slot = e[0]
+                e[0] += size
+                e[1] -= size
+                return slot
+        raise PlanError("POOL_FULL", f"no extent fits {size} slots")
+
     for c in range(n):
         bs = c_bs[c]
-        npg = -(-c_len[c] // bs)
+        if bs:
+            sizes = [bs] * (-(-c_len[c] // bs))
+        else:  # adaptive: the span in 128-slot pages, its tail in 16-slot pages
+            tail = c_len[c] % 128
+            sizes = [128] * (c_len[c] // 128) + [16] * (-(-tail // 16))
+        npg = len(sizes)
         c_first_page[c] = len(page_seg)
         c_n_pages[c] = npg
         pinned = -1 if seg_slot_base is None else seg_slot_base[input_of_canon[c]]
+        at = pinned if pinned >= 0 else (take(sum(sizes)) if not bs else -1)  # adaptive: one extent
+        tok = 0
         for i in range(npg):
-            valid = bs if i < npg - 1 else c_len[c] - (npg - 1) * bs
-            if pinned >= 0:
-                slot = pinned + i * bs
-            elif extents is None:
-                slot = bump
-                bump += bs
+            if at >= 0:
+                slot = at
+                at += sizes[i]
             else:
-                slot = -1
-                for e in extents:
-                    if e[1] >= bs:
-                        slot = e[0]
-                        e[0] += bs
-                        e[1] -= bs
-                        break
-                if slot < 0:
-                    raise PlanError("POOL_FULL", f"no extent fits a page of {bs}")
+                slot = take(sizes[i])
             page_seg.append(c)
-            page_bs.append(bs)
-            page_valid.append(valid)
-            page_pos.append(c_anc[c] + i * bs)
+            page_bs.append(sizes[i])
+            page_valid.append(min(sizes[i], c_len[c] - tok))
+            page_pos.append(c_anc[c] + tok)
             page_ref.append(c_ref[c])
             page_slot.append(slot)
+            tok += sizes[i]
     n_pages = len(page_seg)
     pool_slots = max(page_slot[p] + page_bs[p] for p in range(n_pages))
 
@@ -230,9 +245,11 @@ def oracle_plan(parent, seg_len, group_block_size, seg_flags=None, free_extents=
     # -- step 7: token -> slot ---------------------------------------------------
     tok_slot = [0] * T
     for c in range(n):
-        bs = c_bs[c]
-        for i in range(c_len[c]):
-            tok_slot[c_tok_off[c] + i] = page_slot[c_first_page[c] + i // bs] + i % bs
+        i = 0
+        for pg in range(c_first_page[c], c_first_page[c] + c_n_pages[c]):
+            for j in range(page_valid[pg]):
+                tok_slot[c_tok_off[c] + i] = page_slot[pg] + j
+                i += 1
 
     # -- step 8: samples ----------------------------------------------------------
     sample_end_seg = [c for c in range(n) if c_flags[c] & SEG_SAMPLE_END]

@@ -108,7 +108,7 @@ psrl_status_t psrl_cache_create(const psrl_cache_desc_t* d, psrl_cache_t** out) 
     if (st == PSRL_OK)
       for (int32_t g = 0; g < d->n_groups; ++g) {
         const int32_t b = d->group_block_size[g];
-        if (b < 16 || b > 256 || (b & (b - 1))) st = PSRL_ERR_BAD_BLOCK_SIZE;
+        if (b != 0 && (b < 16 || b > 256 || (b & (b - 1)))) st = PSRL_ERR_BAD_BLOCK_SIZE;
       }
     if (st == PSRL_OK) {
       c.gbs.assign(d->group_block_size, d->group_block_size + d->n_groups);
@@ -117,7 +117,8 @@ psrl_status_t psrl_cache_create(const psrl_cache_desc_t* d, psrl_cache_t** out) 
       for (int32_t s = 0; s < n; ++s) {
         c.group[s] = c.parent[s] == -1 ? g++ : c.group[c.parent[s]];
         c.bs[s] = c.gbs[c.group[s]];
-        c.extent[s] = (int64_t(c.seg_len[s]) + c.bs[s] - 1) / c.bs[s] * c.bs[s];
+        const int64_t unit = c.bs[s] ? c.bs[s] : 16;   // block size 0 = adaptive: the span at 16-slot granularity
+        c.extent[s] = (int64_t(c.seg_len[s]) + unit - 1) / unit * unit;
         c.stats.total_slots += c.extent[s];
       }
       c.sample_end.assign(n, 0);

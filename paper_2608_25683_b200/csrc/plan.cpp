@@ -90,7 +90,9 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
     P.n_groups = static_cast<int32_t>(roots.size());
     if (desc.n_groups != P.n_groups) return PSRL_ERR_INVALID_ARG;
     for (int32_t g = 0; g < P.n_groups; ++g)
-      if (!pow2_in_range(desc.group_block_size[g])) return PSRL_ERR_BAD_BLOCK_SIZE;
+      if (desc.group_block_size[g] != 0 && !pow2_in_range(desc.group_block_size[g])) return PSRL_ERR_BAD_BLOCK_SIZE;
+    for (int32_t g = 0; g < P.n_groups; ++g)  // adaptive blocks: tensor-core path only
+      if (desc.group_block_size[g] == 0 && desc.dtype != PSRL_BF16) return PSRL_ERR_UNSUPPORTED;
     std::vector<Extent> extents;
     const bool bump = desc.free_extents == nullptr;
     for (int32_t i = 0; i < desc.n_free; ++i) {
@@ -178,38 +180,62 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
     // ---- pages ----
     P.seg_first_page.resize(n); P.seg_n_pages.resize(n);
     int64_t bump_at = 0, pool = 0;
+    auto take = [&](int64_t size) -> int64_t {
+      if (bump) {
+        const int64_t slot = bump_at;
+        bump_at += size;
+        return slot;
+      }
+      for (Extent& e : extents) {
+        if (e.count >= size) {
+          const int64_t slot = e.start;
+          e.start += size;
+          e.count -= size;
+          return slot;
+        }
+      }
+      return -1;
+    };
+    std::vector<int32_t> sizes;
     for (int32_t c = 0; c < n; ++c) {
       const int32_t bs = P.seg_bs[c], len = P.seg_len[c];
-      const int32_t npg = (len + bs - 1) / bs;
+      sizes.clear();
+      int64_t total = 0;
+      if (bs) {
+        sizes.assign((len + bs - 1) / bs, bs);
+      } else {  // adaptive (Sec. 5.1): the span in 128-slot pages, its tail in 16-slot pages, one extent
+        sizes.assign(len / kTile, kTile);
+        sizes.insert(sizes.end(), (len % kTile + 15) / 16, 16);
+      }
+      for (int32_t sz : sizes) total += sz;
+      const int32_t npg = static_cast<int32_t>(sizes.size());
       P.seg_first_page[c] = static_cast<int32_t>(P.page_seg.size());
       P.seg_n_pages[c] = npg;
       const int64_t pinned = desc.seg_slot_base ? desc.seg_slot_base[P.input_of_canon[c]] : -1;
+      int64_t at = pinned;
+      if (at < 0 && !bs) {
+        at = take(total);
+        if (at < 0) return PSRL_ERR_POOL_FULL;
+      }
+      int32_t tok = 0;
       for (int32_t i = 0; i < npg; ++i) {
-        int64_t slot = -1;
-        if (pinned >= 0) {
-          slot = pinned + int64_t(i) * bs;
-        } else if (bump) {
-          slot = bump_at;
-          bump_at += bs;
+        int64_t slot;
+        if (at >= 0) {
+          slot = at;
+          at += sizes[i];
         } else {
-          for (Extent& e : extents) {
-            if (e.count >= bs) {
-              slot = e.start;
-              e.start += bs;
-              e.count -= bs;
-              break;
-            }
-          }
+          slot = take(sizes[i]);
           if (slot < 0) return PSRL_ERR_POOL_FULL;
         }
-        if (slot + bs > INT32_MAX / 2) return PSRL_ERR_SHAPE;
+        if (slot + sizes[i] > INT32_MAX / 2) return PSRL_ERR_SHAPE;
         P.page_seg.push_back(c);
-        P.page_bs.push_back(bs);
-        P.page_valid.push_back(i + 1 < npg ? bs : len - i * bs);
-        P.page_pos.push_back(P.seg_anc_tokens[c] + i * bs);
+        P.page_bs.push_back(sizes[i]);
+        P.page_valid.push_back(std::min(sizes[i], len - tok));
+        P.page_pos.push_back(P.seg_anc_tokens[c] + tok);
         P.page_refcount.push_back(P.seg_refcount[c]);
         P.page_slot.push_back(static_cast<int32_t>(slot));
-        pool = std::max<int64_t>(pool, slot + bs);
+        pool = std::max<int64_t>(pool, slot + sizes[i]);
+        tok += sizes[i];
       }
     }
     P.n_pages = static_cast<int32_t>(P.page_seg.size());
@@ -234,10 +260,10 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
 
     // ---- token -> slot ----
     P.tok_slot.resize(P.T);
-    for (int32_t pg = 0; pg < P.n_pages; ++pg) {
-      const int32_t c = P.page_seg[pg];
-      const int32_t first_tok = P.seg_tok_off[c] + (pg - P.seg_first_page[c]) * P.page_bs[pg];
-      for (int32_t j = 0; j < P.page_valid[pg]; ++j) P.tok_slot[first_tok + j] = P.page_slot[pg] + j;
+    for (int32_t c = 0; c < n; ++c) {
+      int32_t tok = P.seg_tok_off[c];
+      for (int32_t pg = P.seg_first_page[c]; pg < P.seg_first_page[c] + P.seg_n_pages[c]; ++pg)
+        for (int32_t j = 0; j < P.page_valid[pg]; ++j) P.tok_slot[tok++] = P.page_slot[pg] + j;
     }
 
     // ---- samples and statistics ----
@@ -268,7 +294,16 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
         kt.bs = bs;
         kt.seg = c;
         kt.tile_idx = t;
-        if (bs >= kTile) {
+        if (bs == 0) {
+          // adaptive block: full tiles are one 128-slot page, the tail tile a run of 16-slot pages
+          const int32_t full = len / kTile;
+          if (t < full) {
+            kt.bs = kTile; kt.first_page = P.seg_first_page[c] + t; kt.n_pages = 1; kt.row_off = 0; kt.rows_loaded = kTile;
+          } else {
+            kt.bs = 16; kt.first_page = P.seg_first_page[c] + full; kt.n_pages = (kt.n_valid + 15) / 16;
+            kt.row_off = 0; kt.rows_loaded = kt.n_pages * 16;
+          }
+        } else if (bs >= kTile) {
           kt.first_page = P.seg_first_page[c] + tok0 / bs;
           kt.n_pages = 1;
           kt.row_off = tok0 % bs;

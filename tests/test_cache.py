@@ -60,6 +60,11 @@ def test_random_schedules_match_oracle(lib):
         run_both(parent, seg_len, gbs, mb, M, flags, cap)
 
 
+def test_adaptive_extents(lib):
+    s = run_both([-1, 0, 0], [28, 4, 300], [0], [0, 0, 1], 2)
+    assert s["total_slots"] == 32 + 16 + 304
+
+
 def test_interleaved_groups(lib):
     s = run_both([-1, 0, 0, -1, 3, 3], [128, 64, 64, 128, 64, 64], [64, 64], [0, 0, 2, 1, 1, 3], 4, cap=192)
     assert s["evicted_slots"] == 256 and s["reloaded_slots"] == 256

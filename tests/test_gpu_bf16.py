@@ -54,6 +54,13 @@ def test_every_block_size(lib, bs):
     check(lib, Workload("b", [-1, 0, 0], [333, 200, 45], [bs], 4, 2, 128, "bf16"), seed=3 + bs, extra_capacity=32)
 
 
+def test_adaptive_blocks(lib):
+    """Block size 0: one extent per segment sized to its span (Sec. 5.1); NaN in every slot that holds
+    no token, next to mixed fixed-size groups."""
+    check(lib, Workload("aba", [-1, 0, 0, 1], [333, 200, 45, 129], [0], 4, 2, 128, "bf16"), seed=71, extra_capacity=32)
+    check(lib, Workload("aba2", [-1, 0, -1, 2, 2], [28, 4, 700, 16, 1], [0, 64], 8, 2, 128, "bf16"), seed=72)
+
+
 def test_odd_group_and_mha(lib):
     # G = 3: one head pair + one single head per KV head; G = 1: MHA
     check(lib, Workload("g3", [-1, 0, 0], [150, 90, 260], [32], 6, 2, 128, "bf16"), seed=5)

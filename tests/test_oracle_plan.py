@@ -203,3 +203,29 @@ def test_synthetic_configs_land_in_paper_ranges():
         p = oracle_plan(w.parent, w.seg_len, w.group_block_size, w.seg_flags, w.free_extents)
         pmr = 1 - p["T"] / p["flat_tokens"]
         assert lo <= pmr <= hi, (name, pmr)
+
+
+def test_adaptive_blocks():
+    """Block size 0 = Adaptive Block Allocation (Sec. 5.1): every segment gets one extent sized to its
+    span at 16-slot granularity, so a 28-token shared span costs 32 slots whatever the page size of
+    other groups, tokens sit at consecutive slots, and the pool is the sum of the rounded spans."""
+    parent, seg_len = [-1, 0, 0, -1, 3], [28, 4, 300, 129, 16]
+    p = oracle_plan(parent, seg_len, [0, 0])
+    ceil16 = lambda x: -(-x // 16) * 16
+    assert p["pool_slots"] == sum(ceil16(l) for l in seg_len)
+    assert int(p["page_valid"].sum()) == sum(seg_len)
+    for c in range(p["n_seg"]):
+        t0, l = int(p["seg_tok_off"][c]), int(p["seg_len"][c])
+        slots = p["tok_slot"][t0:t0 + l]
+        assert np.array_equal(slots, slots[0] + np.arange(l))                 # one contiguous extent
+        sizes = p["page_bs"][p["seg_first_page"][c]:p["seg_first_page"][c] + p["seg_n_pages"][c]].tolist()
+        assert sizes == [128] * (l // 128) + [16] * (-(-(l % 128) // 16))
+    assert p["seg_bs"].tolist() == [0] * 5
+    # the shared 28-token span of the paper's example: 32 slots, stored once, whereas a fixed page of
+    # 32 in a layout that pages whole sequences could not share it (Sec. 5.1)
+    c0 = int(p["canon_of_input"][0])
+    assert int(p["page_bs"][p["seg_first_page"][c0]]) == 16 and int(p["seg_n_pages"][c0]) == 2
+    # mixed with a fixed-size group, fragmented pool: an adaptive extent is taken whole from one free extent
+    q = oracle_plan([-1, -1], [200, 100], [0, 64], None, [(0, 128), (1024, 512)])
+    assert q["page_slot"].tolist()[:3] == [1024, 1152, 1168]     # 200 -> 208 slots do not fit in the first extent
+    assert q["page_slot"].tolist()[6:] == [0, 64]                # the 64-slot pages of the second group do

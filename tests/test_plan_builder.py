@@ -175,3 +175,23 @@ def test_pinned_segments_bit_exact(lib):
     with pytest.raises(lib.PsrlError) as e2:
         lib.Plan([-1, 0], [20, 5], [16], 4, 2, 128, "bf16", seg_slot_base=[8, -1])
     assert e2.value.name == "PSRL_ERR_INVALID_ARG"
+
+
+def test_adaptive_blocks_bit_exact(lib):
+    rng = np.random.default_rng(99)
+    for it in range(30):
+        n_roots = 1 + it % 3
+        parent, seg_len, gbs, flags = random_forest(rng, int(rng.integers(n_roots, 14)), 500, n_roots,
+                                                    block_sizes=(0, 0, 16, 64, 256), cached_roots=(it % 4 == 0))
+        fe = None
+        if it % 3 == 2:
+            fe = [(4096 * i, 2048) for i in range(8)]
+        want = oracle_plan(parent, seg_len, gbs, flags, fe)
+        got = lib.Plan(parent, seg_len, gbs, 4, 2, 128, "bf16", seg_flags=flags, free_extents=fe).view
+        for name in PLAN_ARRAYS:
+            assert np.array_equal(got[name], want[name]), name
+        for name in PLAN_SCALARS:
+            assert int(got[name]) == int(want[name]), name
+    with pytest.raises(lib.PsrlError) as e:     # adaptive blocks exist on the tensor-core path only
+        lib.Plan([-1], [40], [0], 2, 2, 64, "f32")
+    assert e.value.name == "PSRL_ERR_UNSUPPORTED"

@@ -162,6 +162,8 @@ def test_schedule_covers_tree_small_cases(lib):
     check_schedule(small_plan([-1], [300], [16]))
     # two groups with different page sizes
     check_schedule(small_plan([-1, 0, -1, 2, 2], [70, 20, 129, 1, 256], [16, 256]))
+    # adaptive blocks
+    check_schedule(small_plan([-1, 0, 0, 1], [200, 130, 7, 300], [0]))
 
 
 def test_short_suffixes_are_packed_and_split(lib):
