@@ -407,6 +407,10 @@ def main():
     ap.add_argument("--ref-samples", type=int, default=2, help="samples per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unshared", action="store_true")
+    ap.add_argument("--block-size", default=None,
+                    help="override the page size of every group: 16|32|64|128|256, or 'adaptive' (one extent per span)")
+    ap.add_argument("--length-scale", type=float, default=1.0,
+                    help="scale every segment length (tree shape and prefix match rate unchanged, cf. Sec. 7.5)")
     ap.add_argument("--microbatch", action="store_true",
                     help="also run the group as one micro-batch per branch with the Dynamic Block Caching manager")
     args = ap.parse_args()
@@ -432,7 +436,11 @@ def main():
     build.build()
 
     # every rank gets an independent batch of the same shape (groups never span workers)
-    w = make_workload(args.config, dist_util.rank_seed(args.seed, rank))
+    w = make_workload(args.config, dist_util.rank_seed(args.seed, rank), scale_len=args.length_scale)
+    if args.block_size is not None:
+        bs = 0 if args.block_size == "adaptive" else int(args.block_size)
+        w.group_block_size = [bs] * len(w.group_block_size)
+        w.free_extents = None
     r = Runner(lib, w, dist_util.rank_seed(args.seed, rank) + 1, device)
     V = r.plan.view
     flops = dedup_flops(w.head_dim, w.n_q_heads, V["tree_pairs"])
@@ -571,7 +579,7 @@ def main():
     line = dict(metric=METRIC, value=round(value, 3), unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=round(ms_max, 4), higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype=("bf16" if w.dtype == "bf16" else "f32"), data="synthetic",
-                config=dict(workload_config(w, V), l2=(
+                config=dict(workload_config(w, V), length_scale=args.length_scale, pool_slots=V["pool_slots"], l2=(
                     "per-step working set exceeds the 126 MB L2 (inputs larger than L2); no explicit flush" if flush is None
                     else "working set fits in the L2: a 252 MB buffer is overwritten before every timed step "
                          "(each step timed on its own, flush outside the timed part)")), clocks=clocks.summary(), e2e=e2e, gpu_launches=(lib.psrl_launch_count(r.plan, False) + lib.psrl_launch_count(r.plan, True)) * args.steps,
