@@ -337,6 +337,78 @@ def flat_runner(lib, r, device, head_slice=None):
     return Runner(lib, fw, 0, device, data=(q, k, v, d_o))
 
 
+def forest_of_groups(w, groups):
+    """The sub-forest of `w` made of the prefix groups `groups` (root indices counted in input order)."""
+    from paper_2608_25683_b200.workloads import Workload
+
+    root_rank, group_of = -1, []
+    for s, p in enumerate(w.parent):
+        if p == -1:
+            root_rank += 1
+            group_of.append(root_rank)
+        else:
+            group_of.append(group_of[p])
+    keep = [s for s in range(len(w.parent)) if group_of[s] in set(groups)]
+    new = {s: i for i, s in enumerate(keep)}
+    parent = [-1 if w.parent[s] == -1 else new[w.parent[s]] for s in keep]
+    gbs = [w.group_block_size[group_of[s]] for s in keep if w.parent[s] == -1]
+    return Workload(w.name + "-part", parent, [w.seg_len[s] for s in keep], gbs, w.n_q_heads, w.n_kv_heads, w.head_dim,
+                    w.dtype, seed=w.seed)
+
+
+def schedule_leg(lib, device, seed):
+    """Eq. 1 in practice (Sec. 4.2).  (1) The coefficients are fitted by least squares to measured forward +
+    backward times of single prefix groups of varied shape.  (2) The 32 groups of c4 are placed on k workers
+    by descending workload (psrl_place_groups) and, for comparison, round-robin in input order; every worker's
+    share is then run on this GPU and timed: the imbalance is max / mean of the workers' measured times."""
+    from paper_2608_25683_b200.workloads import Workload, make_workload
+
+    Hq, Hkv, d = 32, 8, 128
+    rng = np.random.default_rng(seed)
+
+    def measure(w):
+        r = Runner(lib, w, seed, device)
+        t = time_region(r.step, 5, 2)
+        del r
+        return t
+
+    # ---- (1) fit: T(group) = a1 * sum(l_suf * l) + a2 * sum(l_suf) + a3 * n_samples ----
+    rows, times = [], []
+    for prefix, n_br, br in ((512, 2, 256), (2048, 4, 512), (4096, 8, 512), (8192, 4, 1024), (1024, 16, 128),
+                             (16384, 2, 2048), (256, 8, 1024), (4096, 1, 4096), (12288, 8, 256)):
+        parent = [-1] + [0] * n_br
+        seg_len = [prefix] + [int(br * (0.75 + 0.5 * rng.random())) for _ in range(n_br)]
+        w = Workload("fit", parent, seg_len, [64], Hq, Hkv, d, "bf16", seed=seed)
+        a = [lib.psrl_group_workloads(parent, seg_len, e)[0] for e in ((1, 0, 0), (0, 1, 0), (0, 0, 1))]
+        rows.append(a)
+        times.append(measure(w))
+    A, t = np.asarray(rows), np.asarray(times)
+    alpha, *_ = np.linalg.lstsq(A, t, rcond=None)
+    alpha = np.maximum(alpha, 0.0)
+    fit_err = float(np.max(np.abs(A @ alpha - t) / t))
+
+    # ---- (2) placement of c4's groups ----
+    w = make_workload("c4", 2000)
+    w.free_extents = None
+    workload = lib.psrl_group_workloads(w.parent, w.seg_len, alpha)
+    n_groups = len(workload)
+    out = {"alpha_ms": [float(a) for a in alpha], "fit_max_rel_err": round(fit_err, 4), "n_groups": n_groups, "workers": {}}
+    for k in (2, 4, 8):
+        lpt, load = lib.psrl_place_groups(workload, k)
+        rr = np.arange(n_groups) % k
+        res = {}
+        for name, assign in (("load_balanced", lpt), ("round_robin", rr)):
+            ms = []
+            for worker in range(k):
+                groups = [g for g in range(n_groups) if assign[g] == worker]
+                ms.append(measure(forest_of_groups(w, groups)) if groups else 0.0)
+            pred = [float(sum(workload[g] for g in range(n_groups) if assign[g] == worker)) for worker in range(k)]
+            res[name] = {"measured_ms": [round(x, 2) for x in ms], "predicted_ms": [round(x, 2) for x in pred],
+                         "imbalance_max_over_mean": round(max(ms) / (sum(ms) / k), 4)}
+        out["workers"][str(k)] = res
+    return out
+
+
 def microbatch_leg(lib, w, device, flops, seed, iters):
     """The same forest run as an ordered list of micro-batches (Sec. 4.1): every root is computed with its
     first child, every further child of a root in a micro-batch of its own (deeper levels follow their
@@ -411,6 +483,8 @@ def main():
                     help="override the page size of every group: 16|32|64|128|256, or 'adaptive' (one extent per span)")
     ap.add_argument("--length-scale", type=float, default=1.0,
                     help="scale every segment length (tree shape and prefix match rate unchanged, cf. Sec. 7.5)")
+    ap.add_argument("--schedule", action="store_true",
+                    help="also fit Eq. 1 to measured times and compare load-balanced with round-robin group placement")
     ap.add_argument("--microbatch", action="store_true",
                     help="also run the group as one micro-batch per branch with the Dynamic Block Caching manager")
     args = ap.parse_args()
@@ -568,6 +642,10 @@ def main():
         except Exception as ex:  # e.g. out of memory on the flattened tensors
             unshared = {"error": str(ex)[:200]}
 
+    sched = None
+    if args.schedule and world == 1:
+        sched = schedule_leg(lib, device, args.seed + 11)
+
     micro = None
     if args.microbatch and world == 1:
         micro = microbatch_leg(lib, w, device, flops, args.seed + 7, max(3, min(args.steps, 10)))
@@ -583,7 +661,7 @@ def main():
                     "per-step working set exceeds the 126 MB L2 (inputs larger than L2); no explicit flush" if flush is None
                     else "working set fits in the L2: a 252 MB buffer is overwritten before every timed step "
                          "(each step timed on its own, flush outside the timed part)")), clocks=clocks.summary(), e2e=e2e, gpu_launches=(lib.psrl_launch_count(r.plan, False) + lib.psrl_launch_count(r.plan, True)) * args.steps,
-                roofline=roofline, cpu_baseline=cpu, unshared=unshared, microbatch=micro,
+                roofline=roofline, cpu_baseline=cpu, unshared=unshared, microbatch=micro, schedule=sched,
                 frac_of_bf16_peak={"burst": round(value / world / pk["bf16_tflops"], 4),
                                    "sustained": round(value / world / pk["bf16_tflops_sustained"], 4)})
     print(json.dumps(line), flush=True)

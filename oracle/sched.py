@@ -120,7 +120,10 @@ def microbatch_tokens(parent, seg_len, alpha, n_microbatches, sample_end=None):
     micro-batch `mb`; pieces of one segment are consecutive and form a chain
     (each is the cached prefix of the next)."""
     samples, _ = _samples(parent, seg_len, sample_end)
-    budget = sum(cost_sequence(alpha, l, h) for _, h, l, _ in samples) / n_microbatches
+    total = 0.0
+    for _, h, l, _ in samples:      # plain left-to-right fp64 accumulation (the built-in sum() compensates)
+        total += cost_sequence(alpha, l, h)
+    budget = total / n_microbatches
     pieces = []
     mb, used = 0, 0.0
 

@@ -30,6 +30,7 @@ EXPORTS = [
     "psrl_profile_bwd_phases", "psrl_tree_attn_bwd_static", "psrl_launch_count", "psrl_plan_schedule",
     "psrl_cache_create", "psrl_cache_begin", "psrl_cache_end", "psrl_cache_stats", "psrl_cache_refcounts",
     "psrl_cache_destroy",
+    "psrl_cost_sequence", "psrl_group_workloads", "psrl_place_groups", "psrl_microbatch_tokens",
 ]
 
 _I32P = C.POINTER(C.c_int32)
@@ -42,6 +43,10 @@ class TreeDesc(C.Structure):
         ("head_dim", C.c_int32), ("dtype", C.c_int), ("free_extents", _I32P), ("n_free", C.c_int32),
         ("seg_slot_base", _I32P),
     ]
+
+
+class CostModel(C.Structure):
+    _fields_ = [("a1", C.c_double), ("a2", C.c_double), ("a3", C.c_double)]
 
 
 class CacheDesc(C.Structure):
@@ -135,6 +140,17 @@ def lib() -> C.CDLL:
     L.psrl_profile_bwd_phases.restype = C.c_int
     L.psrl_plan_schedule.argtypes = [C.c_void_p, C.POINTER(_I32P), C.POINTER(C.c_size_t)]
     L.psrl_plan_schedule.restype = C.c_int
+    _F64P = C.POINTER(C.c_double)
+    _U8P = C.POINTER(C.c_uint8)
+    L.psrl_cost_sequence.argtypes = [C.POINTER(CostModel), C.c_int64, C.c_int64]
+    L.psrl_cost_sequence.restype = C.c_double
+    L.psrl_group_workloads.argtypes = [C.c_int32, _I32P, _I32P, _U8P, C.POINTER(CostModel), C.c_int32, _F64P]
+    L.psrl_group_workloads.restype = C.c_int
+    L.psrl_place_groups.argtypes = [C.c_int32, _F64P, C.c_int32, _I32P, _F64P]
+    L.psrl_place_groups.restype = C.c_int
+    L.psrl_microbatch_tokens.argtypes = [C.c_int32, _I32P, _I32P, _U8P, C.POINTER(CostModel), C.c_int32, C.c_int32,
+                                         _I32P, _I32P, _I32P, _I32P, _I32P, _I32P, _F64P]
+    L.psrl_microbatch_tokens.restype = C.c_int
     L.psrl_cache_create.argtypes = [C.POINTER(CacheDesc), C.POINTER(C.c_void_p)]
     L.psrl_cache_create.restype = C.c_int
     L.psrl_cache_begin.argtypes = [C.c_void_p, C.c_int32, C.POINTER(CacheStep)]
@@ -364,6 +380,59 @@ def psrl_profile_bwd_phases(mask: int) -> int:
     """Profiling aid: choose which backward kernels the next calls launch
     (bit 0 delta pre-pass, bit 1 dQ, bit 2 dK/dV); returns the previous mask."""
     return int(lib().psrl_profile_bwd_phases(int(mask)))
+
+
+def _flags_ptr(seg_flags):
+    if seg_flags is None:
+        return None, None
+    fl = np.ascontiguousarray(np.asarray(seg_flags, dtype=np.uint8))
+    return fl, fl.ctypes.data_as(C.POINTER(C.c_uint8))
+
+
+def psrl_cost_sequence(alpha, l: int, h: int) -> float:
+    """Eq. 1 for one sequence of length l with a cached prefix of h tokens."""
+    m = CostModel(*[float(a) for a in alpha])
+    return float(lib().psrl_cost_sequence(C.byref(m), int(l), int(h)))
+
+
+def psrl_group_workloads(parent, seg_len, alpha, seg_flags=None):
+    """Workload of every prefix group (sum of Eq. 1 over its samples)."""
+    p, l = _i32(parent), _i32(seg_len)
+    n_groups = int((p == -1).sum())
+    out = np.zeros(n_groups, dtype=np.float64)
+    m = CostModel(*[float(a) for a in alpha])
+    keep, fp = _flags_ptr(seg_flags)
+    _check(lib().psrl_group_workloads(len(p), p.ctypes.data_as(_I32P), l.ctypes.data_as(_I32P), fp, C.byref(m), n_groups,
+                                      out.ctypes.data_as(C.POINTER(C.c_double))), "psrl_group_workloads")
+    return out
+
+
+def psrl_place_groups(workload, n_workers: int):
+    """Longest-processing-time-first placement: (worker of every group, load of every worker)."""
+    w = np.ascontiguousarray(np.asarray(workload, dtype=np.float64))
+    worker = np.zeros(len(w), dtype=np.int32)
+    load = np.zeros(int(n_workers), dtype=np.float64)
+    _check(lib().psrl_place_groups(len(w), w.ctypes.data_as(C.POINTER(C.c_double)), int(n_workers),
+                                   worker.ctypes.data_as(_I32P), load.ctypes.data_as(C.POINTER(C.c_double))),
+           "psrl_place_groups")
+    return worker, load
+
+
+def psrl_microbatch_tokens(parent, seg_len, alpha, n_microbatches: int, seg_flags=None):
+    """Token-wise micro-batching: the forest of pieces as a dict of arrays (parent, seg_len, mb, seg, begin)
+    plus the per-micro-batch budget."""
+    p, l = _i32(parent), _i32(seg_len)
+    cap = len(p) + int(n_microbatches)
+    outs = [np.zeros(cap, dtype=np.int32) for _ in range(5)]
+    n, budget = C.c_int32(), C.c_double()
+    m = CostModel(*[float(a) for a in alpha])
+    keep, fp = _flags_ptr(seg_flags)
+    _check(lib().psrl_microbatch_tokens(len(p), p.ctypes.data_as(_I32P), l.ctypes.data_as(_I32P), fp, C.byref(m),
+                                        int(n_microbatches), cap, C.byref(n), *[o.ctypes.data_as(_I32P) for o in outs],
+                                        C.byref(budget)), "psrl_microbatch_tokens")
+    k = n.value
+    return dict(parent=outs[0][:k].copy(), seg_len=outs[1][:k].copy(), mb=outs[2][:k].copy(), seg=outs[3][:k].copy(),
+                begin=outs[4][:k].copy(), budget=float(budget.value))
 
 
 class Cache:

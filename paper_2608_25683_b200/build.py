@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsrl.so")
-SOURCES = ["plan.cpp", "cache.cpp", "api.cu", "attn_f32.cu", "attn_bf16_fwd.cu", "attn_bf16_bwd.cu", "attn_bf16_dq.cu", "attn_bf16_dkv.cu", "attn_bf16_merge.cu", "tma.cu", "bwd_static.cu"]
+SOURCES = ["plan.cpp", "cache.cpp", "sched.cpp", "api.cu", "attn_f32.cu", "attn_bf16_fwd.cu", "attn_bf16_bwd.cu", "attn_bf16_dq.cu", "attn_bf16_dkv.cu", "attn_bf16_merge.cu", "tma.cu", "bwd_static.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--expt-relaxed-constexpr",
@@ -22,6 +22,7 @@ def _stale() -> bool:
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
     deps.append(os.path.join(HERE, "..", "include", "psrl.h"))
     deps.append(os.path.join(HERE, "..", "include", "psrl_cache.h"))
+    deps.append(os.path.join(HERE, "..", "include", "psrl_sched.h"))
     deps.append(os.path.abspath(__file__))
     return any(os.path.getmtime(d) > t for d in deps)
 

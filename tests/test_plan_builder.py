@@ -91,7 +91,7 @@ def test_errors_match_oracle(lib):
 
 
 def test_library_exports_every_declared_symbol(lib):
-    hdr = open(os.path.join(ROOT, "include", "psrl.h")).read() + open(os.path.join(ROOT, "include", "psrl_cache.h")).read()
+    hdr = open(os.path.join(ROOT, "include", "psrl.h")).read() + open(os.path.join(ROOT, "include", "psrl_cache.h")).read() + open(os.path.join(ROOT, "include", "psrl_sched.h")).read()
     declared = set(re.findall(r"\b(psrl_[a-z_0-9]+)\s*\(", hdr))
     assert declared, "no declarations found"
     L = lib.lib()
