@@ -483,6 +483,7 @@ def main():
                     help="override the page size of every group: 16|32|64|128|256, or 'adaptive' (one extent per span)")
     ap.add_argument("--length-scale", type=float, default=1.0,
                     help="scale every segment length (tree shape and prefix match rate unchanged, cf. Sec. 7.5)")
+    ap.add_argument("--pack", action="store_true", help="also time K/V scatter into the pools and the gather back")
     ap.add_argument("--schedule", action="store_true",
                     help="also fit Eq. 1 to measured times and compare load-balanced with round-robin group placement")
     ap.add_argument("--microbatch", action="store_true",
@@ -642,6 +643,21 @@ def main():
         except Exception as ex:  # e.g. out of memory on the flattened tensors
             unshared = {"error": str(ex)[:200]}
 
+    pack = None
+    if args.pack and world == 1:
+        import torch as _t
+        T, cap = V["T"], r.k.shape[1]
+        k_tok = _t.randn(T, w.n_kv_heads, w.head_dim, device=device).to(r.k.dtype)
+        v_tok = _t.randn(T, w.n_kv_heads, w.head_dim, device=device).to(r.k.dtype)
+        nbytes_pack = 2 * 2 * k_tok.numel() * k_tok.element_size()      # K and V, read + write
+        fl = device if nbytes_pack < 2 * L2_BYTES else None
+        t_sc = time_region(lambda: lib.psrl_kv_scatter(r.plan, k_tok, v_tok, r.k, r.v), 10, 2, fl)
+        t_ga = time_region(lambda: lib.psrl_kv_gather(r.plan, r.k, r.v, k_tok, v_tok), 10, 2, fl)
+        pack = {"bytes_per_call": nbytes_pack, "scatter_ms": round(t_sc, 4), "gather_ms": round(t_ga, 4),
+                "scatter_gbs": round(nbytes_pack / (t_sc * 1e-3) / 1e9, 1), "gather_gbs": round(nbytes_pack / (t_ga * 1e-3) / 1e9, 1),
+                "hbm_peak_gbs": pk["hbm_gbs"], "scatter_frac": round(nbytes_pack / (t_sc * 1e-3) / 1e9 / pk["hbm_gbs"], 4),
+                "gather_frac": round(nbytes_pack / (t_ga * 1e-3) / 1e9 / pk["hbm_gbs"], 4)}
+
     sched = None
     if args.schedule and world == 1:
         sched = schedule_leg(lib, device, args.seed + 11)
@@ -661,7 +677,7 @@ def main():
                     "per-step working set exceeds the 126 MB L2 (inputs larger than L2); no explicit flush" if flush is None
                     else "working set fits in the L2: a 252 MB buffer is overwritten before every timed step "
                          "(each step timed on its own, flush outside the timed part)")), clocks=clocks.summary(), e2e=e2e, gpu_launches=(lib.psrl_launch_count(r.plan, False) + lib.psrl_launch_count(r.plan, True)) * args.steps,
-                roofline=roofline, cpu_baseline=cpu, unshared=unshared, microbatch=micro, schedule=sched,
+                roofline=roofline, cpu_baseline=cpu, unshared=unshared, microbatch=micro, schedule=sched, kv_pack=pack,
                 frac_of_bf16_peak={"burst": round(value / world / pk["bf16_tflops"], 4),
                                    "sustained": round(value / world / pk["bf16_tflops_sustained"], 4)})
     print(json.dumps(line), flush=True)

@@ -258,6 +258,21 @@ psrl_status_t psrl_tree_attn_bwd_static(const psrl_plan_t* plan, const void* q, 
 psrl_status_t psrl_device_status(const void* workspace, void* stream);
 
 /*
+ * psrl_kv_scatter / psrl_kv_gather - the neighbours of the attention calls: K and V leave the
+ * projections token-major, the attention reads them through the paged pools (Sec. 6, KV manager), and
+ * the gradients of the pools go back token-major.  scatter writes token t of the plan's tree (canonical
+ * order, rows of `k_tok` / `v_tok`) to slot tok_slot[t] of every KV head; gather is the inverse read.
+ * Slots that hold no token are neither written (scatter) nor read (gather).
+ *   k_tok, v_tok  [T, Hkv, d] DEVICE, plan dtype, 16-byte aligned (either pair member may be NULL: skipped)
+ *   k_pool, v_pool [Hkv, pool_capacity, d] DEVICE
+ * Errors: INVALID_ARG, SHAPE, WORKSPACE (plan not uploaded), CUDA.  Asynchronous on `stream`.
+ */
+psrl_status_t psrl_kv_scatter(const psrl_plan_t* plan, const void* k_tok, const void* v_tok, void* k_pool,
+                              void* v_pool, int64_t pool_capacity, void* stream);
+psrl_status_t psrl_kv_gather(const psrl_plan_t* plan, const void* k_pool, const void* v_pool,
+                             int64_t pool_capacity, void* k_tok, void* v_tok, void* stream);
+
+/*
  * Profiling aid (no counterpart in the paper): restricts which kernels the
  * NEXT psrl_tree_attn_bwd calls of this process launch, so that each backward
  * kernel can be timed on its own with CUDA events.  Bit 0: D = rowsum(dO o O)

@@ -30,6 +30,7 @@ EXPORTS = [
     "psrl_profile_bwd_phases", "psrl_tree_attn_bwd_static", "psrl_launch_count", "psrl_plan_schedule",
     "psrl_cache_create", "psrl_cache_begin", "psrl_cache_end", "psrl_cache_stats", "psrl_cache_refcounts",
     "psrl_cache_destroy",
+    "psrl_kv_scatter", "psrl_kv_gather",
     "psrl_cost_sequence", "psrl_group_workloads", "psrl_place_groups", "psrl_microbatch_tokens",
 ]
 
@@ -151,6 +152,10 @@ def lib() -> C.CDLL:
     L.psrl_microbatch_tokens.argtypes = [C.c_int32, _I32P, _I32P, _U8P, C.POINTER(CostModel), C.c_int32, C.c_int32,
                                          _I32P, _I32P, _I32P, _I32P, _I32P, _I32P, _F64P]
     L.psrl_microbatch_tokens.restype = C.c_int
+    L.psrl_kv_scatter.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
+    L.psrl_kv_scatter.restype = C.c_int
+    L.psrl_kv_gather.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.psrl_kv_gather.restype = C.c_int
     L.psrl_cache_create.argtypes = [C.POINTER(CacheDesc), C.POINTER(C.c_void_p)]
     L.psrl_cache_create.restype = C.c_int
     L.psrl_cache_begin.argtypes = [C.c_void_p, C.c_int32, C.POINTER(CacheStep)]
@@ -380,6 +385,41 @@ def psrl_profile_bwd_phases(mask: int) -> int:
     """Profiling aid: choose which backward kernels the next calls launch
     (bit 0 delta pre-pass, bit 1 dQ, bit 2 dK/dV); returns the previous mask."""
     return int(lib().psrl_profile_bwd_phases(int(mask)))
+
+
+def _stream_ptr(stream):
+    import torch
+
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def psrl_kv_scatter(plan: Plan, k_tok, v_tok, k_pool, v_pool, stream=None):
+    """Token-major K, V [T, Hkv, d] -> slots tok_slot[t] of the pools [Hkv, capacity, d] (in place)."""
+    _check_dtype(plan, k_tok, v_tok, k_pool, v_pool)
+    T, Hkv, d = plan.view["T"], plan.n_kv_heads, plan.head_dim
+    for t in (k_tok, v_tok):
+        if tuple(t.shape) != (T, Hkv, d) or not t.is_contiguous():
+            raise ValueError("k_tok / v_tok must be contiguous [T, Hkv, d]")
+    if k_pool.shape != v_pool.shape or k_pool.shape[0] != Hkv or k_pool.shape[2] != d or not k_pool.is_contiguous():
+        raise ValueError("pools must be contiguous [Hkv, capacity, d]")
+    _check(lib().psrl_kv_scatter(plan._h, k_tok.data_ptr(), v_tok.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(),
+                                 int(k_pool.shape[1]), _stream_ptr(stream)), "psrl_kv_scatter")
+
+
+def psrl_kv_gather(plan: Plan, k_pool, v_pool, k_tok=None, v_tok=None, stream=None):
+    """The inverse read: pools -> token-major [T, Hkv, d] (e.g. dK, dV back to the projections)."""
+    import torch
+
+    _check_dtype(plan, k_pool, v_pool)
+    T, Hkv, d = plan.view["T"], plan.n_kv_heads, plan.head_dim
+    if k_tok is None:
+        k_tok = torch.empty((T, Hkv, d), dtype=k_pool.dtype, device=k_pool.device)
+    if v_tok is None:
+        v_tok = torch.empty((T, Hkv, d), dtype=v_pool.dtype, device=v_pool.device)
+    _check(lib().psrl_kv_gather(plan._h, k_pool.data_ptr(), v_pool.data_ptr(), int(k_pool.shape[1]), k_tok.data_ptr(),
+                                v_tok.data_ptr(), _stream_ptr(stream)), "psrl_kv_gather")
+    return k_tok, v_tok
 
 
 def _flags_ptr(seg_flags):

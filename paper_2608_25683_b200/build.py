@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsrl.so")
-SOURCES = ["plan.cpp", "cache.cpp", "sched.cpp", "api.cu", "attn_f32.cu", "attn_bf16_fwd.cu", "attn_bf16_bwd.cu", "attn_bf16_dq.cu", "attn_bf16_dkv.cu", "attn_bf16_merge.cu", "tma.cu", "bwd_static.cu"]
+SOURCES = ["plan.cpp", "cache.cpp", "sched.cpp", "api.cu", "attn_f32.cu", "attn_bf16_fwd.cu", "attn_bf16_bwd.cu", "attn_bf16_dq.cu", "attn_bf16_dkv.cu", "attn_bf16_merge.cu", "tma.cu", "bwd_static.cu", "kv_pack.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--expt-relaxed-constexpr",

@@ -524,6 +524,7 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
     H.off_bt_off = append_array(B, P.bt_off);
     H.off_bt_pages = append_array(B, P.bt_pages);
     H.off_qrow_seg = append_array(B, P.qrow_seg);
+    H.off_tok_slot = append_array(B, P.tok_slot);
     H.off_kvt = append_array(B, P.kv_tiles);
     H.off_qt = append_array(B, P.q_tiles);
     H.off_kvi = append_array(B, P.kv_items);

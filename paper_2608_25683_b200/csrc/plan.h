@@ -98,7 +98,7 @@ struct DeviceHeader {
   // merge lists of the rows that are assembled from partial results: row i of the list is
   // query row merge_row[i]; its parts are merge_parts[merge_off[i] .. merge_off[i+1]) (partial-row ids)
   int32_t n_part_rows, n_merge_rows, off_merge_row, off_merge_off, off_merge_parts;
-  int32_t reserved[1];
+  int32_t off_tok_slot;     // [T] pool slot of every token
 };
 
 struct Plan {
