@@ -17,8 +17,8 @@
 // a step ready, fetch them in one tensor-memory round trip and compute P and dS
 // element by element in one pass.
 //
-// Warp roles: warps 0-7 softmax-backward (two threads per query row, 64 keys
-// each), warp 8 TMA producer, warp 9 MMA issuer + TMEM owner.
+// Warp roles: warps 0-3 softmax-backward (one query row per thread), warp 4 TMA
+// producer, warp 5 MMA issuer + TMEM owner.
 // Tensor memory: S at 0, dP / dS at 128 and 256 (alternating), dQ at 384.
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -32,7 +32,8 @@ namespace {
 using namespace sm100;
 
 constexpr int KS = 3, VS = 2;                 // K and V ring depths
-constexpr int kThreads = (8 + 2) * 32;
+constexpr int kSW = 4;                        // softmax-backward warps: one per SM sub-partition
+constexpr int kThreads = (kSW + 2) * 32;
 constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 384;   // dP / dS is double-buffered: 128 and 256
 
 struct Maps {
@@ -79,19 +80,19 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     mbar_init(&bar.qdo_full, 1);
     for (int i = 0; i < KS; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1); }
     for (int i = 0; i < VS; ++i) { mbar_init(&bar.v_full[i], 1); mbar_init(&bar.v_empty[i], 1); }
-    mbar_init(&bar.s_full, 1); mbar_init(&bar.s_free, 256);
-    for (int i = 0; i < 2; ++i) { mbar_init(&bar.dp_full[i], 1); mbar_init(&bar.ds_ready[i], 256); }
+    mbar_init(&bar.s_full, 1); mbar_init(&bar.s_free, kSW * 32);
+    for (int i = 0; i < 2; ++i) { mbar_init(&bar.dp_full[i], 1); mbar_init(&bar.ds_ready[i], kSW * 32); }
     mbar_init(&bar.dq_done, 1);
     fence_mbar_init();
   }
-  if (warp == 9) { tmem_alloc(&s_tmem, 512); tmem_relinquish(); }
+  if (warp == kSW + 1) { tmem_alloc(&s_tmem, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   volatile int* abortp = &s_abort;
 
-  if (warp == 8) {
+  if (warp == kSW) {
     // ======================= TMA producer =======================
     if (lane == 0) {
       mbar_expect_tx(&bar.qdo_full, 2 * kTileBytes);
@@ -114,7 +115,7 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
         cur = nxt;
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == kSW + 1) {
     // ======================= MMA issuer =======================
     // All 32 lanes walk the loop and wait on the barriers (warp-uniform control flow and
     // address arithmetic); only the tcgen05 instructions are issued, by one elected lane.
@@ -176,10 +177,12 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     }
     if (ok) commit(&bar.dq_done);
   } else {
-    // ======================= softmax-backward warps (8) =======================
-    const int half = warp >> 2;                           // which 64 keys of the tile
-    const int row = (warp & 3) * 32 + lane;               // query row inside the tile = TMEM lane
-    const uint32_t t_lane = tmem + (uint32_t((warp & 3) * 32) << 16);
+    // ======================= softmax-backward warps (4) =======================
+    // One warp per SM sub-partition, one query row per thread.  (Two warps per sub-partition
+    // compute a little faster, but between them they take every issue slot, and the MMA and
+    // producer warps that share the sub-partitions then fall behind.)
+    const int row = warp * 32 + lane;                     // query row inside the tile = TMEM lane
+    const uint32_t t_lane = tmem + (uint32_t(warp * 32) << 16);
     const bool row_ok = row < qt.n_rows;
     const float lse2 = row_ok ? p.lse[int64_t(h) * p.T_q + qt.q_row0 + row] * kLog2e : 0.f;
     const float dl = row_ok ? p.delta[int64_t(h) * p.T_q + qt.q_row0 + row] : 0.f;
@@ -194,41 +197,50 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       const int limit = diag ? min(row + 1, n_valid) : n_valid;   // keys [0, limit) are visible
       const bool need_mask = diag || n_valid < 128;
       // S(j) and dP(j) are both complete well before the warps get here (the MMA warp issues them
-      // one step ahead), so both are fetched in one round trip; S may then be overwritten.
+      // one step ahead).  The whole score row goes to registers at once, so S may be overwritten.
       const uint32_t t_dp = t_lane + TM_DP + (j & 1) * 128;
       ok = mbar_wait(&bar.s_full, j & 1, abortp, p.status) &&
            mbar_wait(&bar.dp_full[j & 1], (j >> 1) & 1, abortp, p.status);
       if (!ok) break;
       tc_fence_after();
-      uint32_t s[2][32], dp[2][32];
-      tmem_ld32(t_lane + TM_S + half * 64, s[0]);
-      tmem_ld32(t_lane + TM_S + half * 64 + 32, s[1]);
-      tmem_ld32(t_dp + half * 64, dp[0]);
-      tmem_ld32(t_dp + half * 64 + 32, dp[1]);
+      uint32_t s[4][32], dp[2][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(t_lane + TM_S + c * 32, s[c]);
+      tmem_ld32(t_dp, dp[0]);
+      tmem_ld32(t_dp + 32, dp[1]);
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&bar.s_free);
       // P = exp2(S c - LSE) and dS = P o (dP - D) element by element: the exp2 (MUFU pipe) of one
       // element overlaps the arithmetic of its neighbours instead of forming a phase of its own
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int x = 0; x < 32; x += 2) {
-          float a0, a1, d0, d1;
-          split_f32x2(fma2(make_f32x2(s[c][x], s[c][x + 1]), scale2, neg_lse2), a0, a1);
-          const f32x2 pp = make_f32x2(ex2(a0), ex2(a1));
-          split_f32x2(mul2(pp, add2(make_f32x2(dp[c][x], dp[c][x + 1]), neg_dl2)), d0, d1);
-          if (need_mask) {  // masked columns may hold anything (pad rows of K, V): select, do not multiply
-            d0 = (half * 64 + c * 32 + x < limit) ? d0 : 0.f;
-            d1 = (half * 64 + c * 32 + x + 1 < limit) ? d1 : 0.f;
-          }
-          pk[x >> 1] = pack_bf16(d0, d1);
+      for (int half = 0; half < 2; ++half) {
+        if (half == 1) {
+          tmem_ld32(t_dp + 64, dp[0]);
+          tmem_ld32(t_dp + 96, dp[1]);
+          tmem_wait_ld();
         }
-        tmem_st16(t_dp + half * 64 + c * 16, pk);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int x = 0; x < 32; x += 2) {
+            float a0, a1, d0, d1;
+            split_f32x2(fma2(make_f32x2(s[half * 2 + c][x], s[half * 2 + c][x + 1]), scale2, neg_lse2), a0, a1);
+            const f32x2 pp = make_f32x2(ex2(a0), ex2(a1));
+            split_f32x2(mul2(pp, add2(make_f32x2(dp[c][x], dp[c][x + 1]), neg_dl2)), d0, d1);
+            if (need_mask) {  // masked columns may hold anything (pad rows of K, V): select, do not multiply
+              d0 = (half * 64 + c * 32 + x < limit) ? d0 : 0.f;
+              d1 = (half * 64 + c * 32 + x + 1 < limit) ? d1 : 0.f;
+            }
+            pk[x >> 1] = pack_bf16(d0, d1);
+          }
+          // dS: packed bf16, keys 0-63 in columns [0, 32), keys 64-127 in columns [64, 96) of the dP buffer
+          tmem_st16(t_dp + half * 64 + c * 16, pk);
+        }
       }
       // K rows at or beyond n_valid must be zero before dS K (dS is zero there, K may hold anything)
-      if (n_valid < 128 && half == 0) {
+      if (n_valid < 128) {
         ok = mbar_wait(&bar.k_full[j % KS], (j / KS) & 1, abortp, p.status);
         if (!ok) break;
         if (row >= n_valid) zero_tile_row(sK + (j % KS) * kTileBytes, row);
@@ -242,15 +254,15 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     if (ok) ok = mbar_wait(&bar.dq_done, 0, abortp, p.status);
     if (ok) {
       tc_fence_after();
-      __nv_bfloat16* drow = p.d_q + (int64_t(qt.q_row0 + row) * p.Hq + h) * 128 + half * 64;
+      __nv_bfloat16* drow = p.d_q + (int64_t(qt.q_row0 + row) * p.Hq + h) * 128;
 #pragma unroll
-      for (int c = 0; c < 2; ++c) {
+      for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
-        tmem_ld32(t_lane + TM_DQ + half * 64 + c * 32, r);
+        tmem_ld32(t_lane + TM_DQ + c * 32, r);
         tmem_wait_ld();
         if (row_ok && qt.part_row0 >= 0) {
           // the row has other contributors: unscaled fp32 partial, summed by the merge kernel
-          float* prow = p.part + (int64_t(qt.part_row0 + row) * p.Hq + h) * 128 + half * 64 + c * 32;
+          float* prow = p.part + (int64_t(qt.part_row0 + row) * p.Hq + h) * 128 + c * 32;
 #pragma unroll
           for (int x = 0; x < 8; ++x)
             *reinterpret_cast<float4*>(prow + x * 4) =
@@ -272,7 +284,7 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == kSW + 1) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
