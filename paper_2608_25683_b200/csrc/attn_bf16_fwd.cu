@@ -225,8 +225,49 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) tmem_ld32(t_lane + c * 32, s[c]);
       tmem_wait_ld();
+      // exponentials of the row against the reference m, P stored as bf16, row sum returned; with
+      // mx_out the row maximum (raw scores) is tracked in the same pass
+      auto exp_pass = [&](float m, bool masked, float* mx_out) -> float {
+        f32x2 sum2 = make_f32x2(0.f, 0.f);
+        const f32x2 neg_m2 = make_f32x2(-m, -m);
+        float mx = -CUDART_INF_F;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            float a0, a1;
+            split_f32x2(fma2(make_f32x2(s[c][i], s[c][i + 1]), scale2, neg_m2), a0, a1);
+            float e0 = ex2(a0), e1 = ex2(a1);
+            if (masked) {
+              e0 = (c * 32 + i < limit) ? e0 : 0.f;
+              e1 = (c * 32 + i + 1 < limit) ? e1 : 0.f;
+            }
+            if (mx_out) mx = fmax3(mx, __uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1]));
+            sum2 = add2(sum2, make_f32x2(e0, e1));
+            pk[i >> 1] = pack_bf16(e0, e1);
+          }
+          tmem_st16(t_lane + c * 16, pk);
+        }
+        if (mx_out) *mx_out = mx;
+        float lo, hi;
+        split_f32x2(sum2, lo, hi);
+        return lo + hi;
+      };
+      float sum, m_use, alpha;
+      bool any_move;
+      bool settled = false;
       float mx = -CUDART_INF_F;
-      if (need_mask) {
+      if (j > 0 && !need_mask) {
+        // Interior tile: bet that the reference stays (it moves only when the maximum grows by more than
+        // 2^8, rare after the first tiles) and compute the exponentials at once, tracking the maximum on
+        // the side instead of in a pass of its own; if the bet fails for any row of the warp the tile is
+        // redone below (P and the sum are simply recomputed from the scores held in registers).
+        sum = exp_pass(m_ref, false, &mx);
+        const bool move = fmaxf(m_ref, mx * p.scale_log2) > m_ref + 8.f;
+        any_move = __any_sync(0xffffffffu, move);
+        if (!any_move) { settled = true; m_use = m_ref; alpha = 1.f; }
+      } else if (need_mask) {
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
@@ -239,33 +280,14 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
           for (int i = 0; i < 32; i += 2)
             mx = fmax3(mx, __uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1]));
       }
-      const float m_new = fmaxf(m_ref, mx * p.scale_log2);
-      const bool move = m_new > m_ref + 8.f;            // also true on the first tile (m_ref = -inf)
-      const bool any_move = __any_sync(0xffffffffu, move);
-      const float m_use = move ? m_new : m_ref;
-      const float alpha = ex2(m_ref - m_use);            // 1 if the reference stays, 0 on the first tile
-      f32x2 sum2 = make_f32x2(0.f, 0.f);
-      const f32x2 neg_m2 = make_f32x2(-m_use, -m_use);
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          float a0, a1;
-          split_f32x2(fma2(make_f32x2(s[c][i], s[c][i + 1]), scale2, neg_m2), a0, a1);
-          float e0 = ex2(a0), e1 = ex2(a1);
-          if (need_mask) {
-            e0 = (c * 32 + i < limit) ? e0 : 0.f;
-            e1 = (c * 32 + i + 1 < limit) ? e1 : 0.f;
-          }
-          sum2 = add2(sum2, make_f32x2(e0, e1));
-          pk[i >> 1] = pack_bf16(e0, e1);
-        }
-        tmem_st16(t_lane + c * 16, pk);
+      if (!settled) {
+        const float m_new = fmaxf(m_ref, mx * p.scale_log2);
+        const bool move = m_new > m_ref + 8.f;            // also true on the first tile (m_ref = -inf)
+        any_move = __any_sync(0xffffffffu, move);
+        m_use = move ? m_new : m_ref;
+        alpha = ex2(m_ref - m_use);                        // 1 if the reference stays, 0 on the first tile
+        sum = exp_pass(m_use, need_mask, nullptr);
       }
-      float sum_lo, sum_hi;
-      split_f32x2(sum2, sum_lo, sum_hi);
-      const float sum = sum_lo + sum_hi;
       l_run = fmaf(l_run, alpha, sum);
       m_ref = m_use;
       // ---- the reference moved: rescale the accumulated output in tensor memory ----
