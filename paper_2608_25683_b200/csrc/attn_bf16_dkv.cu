@@ -1,7 +1,7 @@
 // bf16 dK/dV kernel (key-stationary) and the fixed-order reduce of split tiles.
 //
 // One CTA = one work item: a KV tile (<= 128 keys of one segment, one KV head)
-// and a range of 64-row query sub-tiles that attend to it - the later rows of
+// and a range of 128-row query sub-tiles that attend to it - the later rows of
 // the tile's own segment, then the rows of ALL descendant segments, which form
 // one contiguous row range in the canonical layout (paper Sec. 6: the adjoints
 // of every consumer are accumulated on the shared prefix) - times the Hq/Hkv
@@ -10,14 +10,17 @@
 //
 // Per step (128 query rows of one head) the tensor cores run four contractions
 // (M = 128 keys, N = 128, K = 128) and the warps run two half-steps:
-//   S^T  = K Q^T                 -> warps: P^T = exp2(S^T c - LSE), written over S^T as bf16
+//   S^T  = K Q^T - LSE/c         -> warps: P^T = exp2(S^T c), written over S^T as bf16
 //   dV  += P^T dO                   (A = P^T from tensor memory, dO MN-major in smem)
-//   dP^T = V dO^T                -> warps: dS^T = P^T o (dP^T - D), written over dP^T as bf16
+//   dP^T = V dO^T - D            -> warps: dS^T = P^T o dP^T, written over dP^T as bf16
 //   dK  += dS^T Q                   (A = dS^T from tensor memory, Q MN-major in smem)
 // The issue order is  dV(i), S^T(i+1), dK(i), dP^T(i+1):  while the warps turn S^T(i+1)
 // into P^T(i+1) the tensor cores work on dK(i) and dP^T(i+1); while they turn dP^T(i+1)
 // into dS^T(i+1) the tensor cores work on dV(i+1) and S^T(i+2).  S^T may be overwritten
 // as soon as dV(i) has been issued (it consumed P^T(i)), dP^T as soon as dK(i) has been.
+//
+// The per-row terms -LSE/c and -D enter S^T and dP^T as one more K = 16 MMA slice (a three-term bf16
+// split of the value against a slice of ones), so the warps need no per-column loads.
 //
 // Tensor memory (512 columns): S^T at 0, dP^T at 128, dV at 256, dK at 384.
 // Heavy tiles are split over several CTAs by the plan; a split item writes its

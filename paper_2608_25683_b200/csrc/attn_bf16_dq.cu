@@ -1,9 +1,9 @@
 // bf16 dQ kernel (query-stationary).
 //
-// One CTA = one query tile (up to 128 rows of one segment) x one query head.
-// It walks the tile's path of KV tiles exactly like the forward (all tiles of
-// the ancestor segments, then the own segment's tiles up to the diagonal) and
-// per tile runs three contractions (M = 128 rows, N = 128, K = 128):
+// One CTA = one work item (up to 128 query rows and a list of KV tiles, see
+// plan.h: the rows of one segment with the tiles of its ancestors and its own
+// tiles up to the diagonal, or packed rows under a cascaded prefix) x one query
+// head.  Per tile it runs three contractions (M = 128 rows, N = 128, K = 128):
 //   S  = Q K^T      -> warps: P = exp2(S c - LSE), kept in registers
 //   dP = dO V^T     -> warps: dS = P o (dP - D), written over dP as bf16
 //   dQ += dS K         (A = dS from tensor memory, K MN-major in smem)
