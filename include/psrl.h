@@ -168,7 +168,8 @@ size_t psrl_bwd_workspace_bytes(const psrl_plan_t* plan);
  * For every query row i of a HAS_Q segment c and query head h (KV head
  * h / (Hq/Hkv)):  keys = all tokens of c's ancestors + tokens 0..i of c;
  *   O_i = softmax_j(scale * q_i . k_j) V,   LSE_i = ln sum_j exp(scale * q_i . k_j).
- * All tensor pointers are DEVICE pointers, 16-byte aligned, dtype = plan dtype:
+ * All tensor pointers are DEVICE pointers, 16-byte aligned, dtype = plan dtype (the Q-shaped ones may
+ * be NULL when the plan has no query row at all, T_q = 0):
  *   q        [T_q, Hq, d]  read only; rows of segment c start at seg_q_off[c]
  *   k_pool   [Hkv, pool_capacity, d] read only; token t lives at slot tok_slot[t]
  *   v_pool   same layout.  Slots that hold no token (page pads, free slots)

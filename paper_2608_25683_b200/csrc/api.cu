@@ -20,6 +20,10 @@ int g_bwd_phase_mask = 7;
 namespace {
 
 bool aligned(const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+// Q-shaped tensors of a plan without any query row are empty: NULL is fine there
+bool aligned_q(const void* p, size_t a, const psrl::Plan& P) {
+  return (P.T_q == 0 && !p) || aligned(p, a);
+}
 
 size_t ws_bytes(const psrl::Plan& P, bool bwd) {
   size_t n = psrl::kWsHeaderBytes;
@@ -113,8 +117,8 @@ psrl_status_t psrl_tree_attn_fwd(const psrl_plan_t* plan, const void* q, const v
                                  size_t workspace_bytes, void* stream) {
   if (!plan || !plan->p) return PSRL_ERR_INVALID_ARG;
   const psrl::Plan& P = *plan->p;
-  if (!aligned(q, 16) || !aligned(k_pool, 16) || !aligned(v_pool, 16) || !aligned(o, 16) || !aligned(lse, 16) ||
-      !aligned(workspace, 256))
+  if (!aligned_q(q, 16, P) || !aligned(k_pool, 16) || !aligned(v_pool, 16) || !aligned_q(o, 16, P) ||
+      !aligned_q(lse, 16, P) || !aligned(workspace, 256))
     return PSRL_ERR_INVALID_ARG;
   if (pool_capacity < P.pool_slots) return PSRL_ERR_SHAPE;
   if (!P.dev || workspace_bytes < ws_bytes(P, false)) return PSRL_ERR_WORKSPACE;
@@ -137,9 +141,9 @@ psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const v
                                  size_t workspace_bytes, void* stream) {
   if (!plan || !plan->p) return PSRL_ERR_INVALID_ARG;
   const psrl::Plan& P = *plan->p;
-  if (!aligned(q, 16) || !aligned(k_pool, 16) || !aligned(v_pool, 16) || !aligned(o, 16) || !aligned(lse, 16) ||
-      !aligned(d_o, 16) || !aligned(d_q, 16) || !aligned(dk_pool, 16) || !aligned(dv_pool, 16) ||
-      !aligned(workspace, 256))
+  if (!aligned_q(q, 16, P) || !aligned(k_pool, 16) || !aligned(v_pool, 16) || !aligned_q(o, 16, P) ||
+      !aligned_q(lse, 16, P) || !aligned_q(d_o, 16, P) || !aligned_q(d_q, 16, P) || !aligned(dk_pool, 16) ||
+      !aligned(dv_pool, 16) || !aligned(workspace, 256))
     return PSRL_ERR_INVALID_ARG;
   if (pool_capacity < P.pool_slots) return PSRL_ERR_SHAPE;
   if (!P.dev || workspace_bytes < ws_bytes(P, true)) return PSRL_ERR_WORKSPACE;

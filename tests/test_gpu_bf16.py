@@ -148,3 +148,26 @@ def test_runs_are_bitwise_reproducible(lib):
             assert torch.equal(a[key], b[key])
         for key in ("dK", "dV"):
             assert torch.equal(torch.nan_to_num(a[key]), torch.nan_to_num(b[key]))
+
+
+def test_no_queries_at_all(lib):
+    """Degenerate input: every segment is a cached prefix (no queries anywhere).  Forward has nothing to
+    write; backward still owns the gradient pools and writes zeros to every slot of every page."""
+    w = Workload("nq", [-1, 0], [200, 70], [64], 4, 2, 128, "bf16", seg_flags=[0, 2])
+    plan = build_plan(lib, w)
+    V = plan.view
+    assert V["T_q"] == 0
+    cap = V["pool_slots"] + 64
+    q = torch.zeros(0, 4, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.randn(2, cap, 128, device="cuda").to(torch.bfloat16)
+    v = torch.randn(2, cap, 128, device="cuda").to(torch.bfloat16)
+    o, lse = lib.psrl_tree_attn_fwd(plan, q, k, v, 0.1)
+    assert o.shape[0] == 0 and lib.psrl_device_status(plan, "fwd") == 0
+    dk = torch.full_like(k, float("nan")); dv = torch.full_like(v, float("nan"))
+    dq, dk, dv = lib.psrl_tree_attn_bwd(plan, q, k, v, o, lse, q, 0.1, dk_pool=dk, dv_pool=dv)
+    assert lib.psrl_device_status(plan, "bwd") == 0
+    tok, padm, outside = page_masks(V, cap)
+    dkn, dvn = to_np(dk), to_np(dv)
+    assert np.all(dkn[:, tok] == 0) and np.all(dvn[:, tok] == 0)
+    assert np.all(dkn[:, padm] == 0) and np.all(dvn[:, padm] == 0)
+    assert np.all(np.isnan(dkn[:, outside]))
