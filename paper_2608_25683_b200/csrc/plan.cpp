@@ -540,6 +540,15 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
       tl = TileLoad{};
       tl.n_pages = kt.n_pages; tl.bs = kt.bs; tl.rows_loaded = kt.rows_loaded;
       for (int32_t pg = 0; pg < kt.n_pages && pg < 8; ++pg) tl.row[pg] = P.page_slot[kt.first_page + pg] + kt.row_off;
+      // Pages that follow one another in the pool (always, under bump allocation) are fetched as ONE box
+      // when together they make a power-of-two number of rows: a TMA box costs ~135 cycles plus its bytes.
+      const int32_t page_rows = kt.bs >= kTile ? kTile : kt.bs;
+      bool contiguous = kt.n_pages > 1;
+      for (int32_t pg = 1; pg < kt.n_pages && contiguous; ++pg) contiguous = tl.row[pg] == tl.row[pg - 1] + page_rows;
+      if (contiguous && (kt.rows_loaded & (kt.rows_loaded - 1)) == 0) {
+        tl.n_pages = 1;
+        tl.bs = kt.rows_loaded;   // 32, 64 or 128: selects the box height
+      }
     }
     H.off_path_loads = append_array(B, P.path_loads);
     H.n_kvi = static_cast<int32_t>(P.kv_items.size());
