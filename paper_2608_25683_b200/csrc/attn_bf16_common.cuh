@@ -43,6 +43,14 @@ __device__ __forceinline__ void load_kv_tile_at(uint8_t* dst, const CUtensorMap*
   const int rows_per_box = tl.bs >= 128 ? 128 : tl.bs;
   const CUtensorMap* m = maps + map_index(tl.bs);
   mbar_expect_tx(bar, uint32_t(tl.rows_loaded) * 256u);
+  if (tl.n_pages == 1) {
+    // the common case (pages contiguous in the pool): one box per half, and as few instructions as
+    // possible - the producer shares its scheduler with two softmax warps
+    const int row = int(head_row0 + tl.row[0]);
+    tma_load_2d(dst, m, bar, 0, row);
+    tma_load_2d(dst + kHalfBytes, m, bar, 64, row);
+    return;
+  }
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     if (i < tl.n_pages) {
