@@ -336,24 +336,36 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
         tmem_ld32(t_lane + TM_ST + wg * 64, s[0]);
         tmem_ld32(t_lane + TM_ST + wg * 64 + 32, s[1]);
         tmem_wait_ld();
+        // software pipeline over groups of 16 query rows: the exp2 of group g+1 (MUFU pipe) is issued
+        // before group g is masked, packed and stored
+        auto exps = [&](int g) {
+          const int c = g >> 1, i0 = (g & 1) * 16;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int x = 0; x < 32; x += 2) {
+          for (int i = 0; i < 16; i += 2) {
             float a0, a1;
-            split_f32x2(mul2(make_f32x2(s[c][x], s[c][x + 1]), scale2), a0, a1);
-            float p0 = ex2(a0), p1 = ex2(a1);
+            split_f32x2(mul2(make_f32x2(s[c][i0 + i], s[c][i0 + i + 1]), scale2), a0, a1);
+            pr[g * 16 + i] = ex2(a0);
+            pr[g * 16 + i + 1] = ex2(a1);
+          }
+        };
+        exps(0);
+        uint32_t pk[16];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          if (g + 1 < 4) exps(g + 1);
+#pragma unroll
+          for (int i = 0; i < 16; i += 2) {
+            float p0 = pr[g * 16 + i], p1 = pr[g * 16 + i + 1];
             if (diag) {  // the tile that holds the keys' own rows: a key is visible from its own row on
-              const int col = wg * 64 + c * 32 + x;
+              const int col = wg * 64 + g * 16 + i;
               p0 = (qpos0 + col >= keyrow) ? p0 : 0.f;
               p1 = (qpos0 + col + 1 >= keyrow) ? p1 : 0.f;
+              pr[g * 16 + i] = p0;
+              pr[g * 16 + i + 1] = p1;
             }
-            pr[c * 32 + x] = p0;
-            pr[c * 32 + x + 1] = p1;
-            pk[x >> 1] = pack_bf16(p0, p1);
+            pk[(g & 1) * 8 + (i >> 1)] = pack_bf16(p0, p1);
           }
-          tmem_st16(t_lane + TM_ST + wg * 64 + c * 16, pk);
+          if (g & 1) tmem_st16(t_lane + TM_ST + wg * 64 + (g >> 1) * 16, pk);
         }
       }
       tmem_wait_st();

@@ -220,23 +220,39 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
           tmem_ld32(t_dp + 96, dp[1]);
           tmem_wait_ld();
         }
+        // software pipeline over groups of 16 keys: the exp2 of group g+1 (MUFU pipe) is issued before
+        // group g is multiplied, packed and stored
+        float pe[2][16];
+        auto exps = [&](int g, float (&out)[16]) {
+          const int c = half * 2 + (g >> 1), i0 = (g & 1) * 16;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t pk[16];
+          for (int i = 0; i < 16; i += 2) {
+            float a0, a1;
+            split_f32x2(fma2(make_f32x2(s[c][i0 + i], s[c][i0 + i + 1]), scale2, neg_lse2), a0, a1);
+            out[i] = ex2(a0);
+            out[i + 1] = ex2(a1);
+          }
+        };
+        exps(0, pe[0]);
+        uint32_t pk[16];
 #pragma unroll
-          for (int x = 0; x < 32; x += 2) {
-            float a0, a1, d0, d1;
-            split_f32x2(fma2(make_f32x2(s[half * 2 + c][x], s[half * 2 + c][x + 1]), scale2, neg_lse2), a0, a1);
-            const f32x2 pp = make_f32x2(ex2(a0), ex2(a1));
-            split_f32x2(mul2(pp, add2(make_f32x2(dp[c][x], dp[c][x + 1]), neg_dl2)), d0, d1);
+        for (int g = 0; g < 4; ++g) {
+          if (g + 1 < 4) exps(g + 1, pe[(g + 1) & 1]);
+          float (&cur)[16] = pe[g & 1];
+          const int c = g >> 1, i0 = (g & 1) * 16;
+#pragma unroll
+          for (int i = 0; i < 16; i += 2) {
+            float d0, d1;
+            split_f32x2(mul2(make_f32x2(cur[i], cur[i + 1]),
+                             add2(make_f32x2(dp[c][i0 + i], dp[c][i0 + i + 1]), neg_dl2)), d0, d1);
             if (need_mask) {  // masked columns may hold anything (pad rows of K, V): select, do not multiply
-              d0 = (half * 64 + c * 32 + x < limit) ? d0 : 0.f;
-              d1 = (half * 64 + c * 32 + x + 1 < limit) ? d1 : 0.f;
+              d0 = (half * 64 + g * 16 + i < limit) ? d0 : 0.f;
+              d1 = (half * 64 + g * 16 + i + 1 < limit) ? d1 : 0.f;
             }
-            pk[x >> 1] = pack_bf16(d0, d1);
+            pk[(g & 1) * 8 + (i >> 1)] = pack_bf16(d0, d1);
           }
           // dS: packed bf16, keys 0-63 in columns [0, 32), keys 64-127 in columns [64, 96) of the dP buffer
-          tmem_st16(t_dp + half * 64 + c * 16, pk);
+          if (g & 1) tmem_st16(t_dp + half * 64 + c * 16, pk);
         }
       }
       // K rows at or beyond n_valid must be zero before dS K (dS is zero there, K may hold anything)

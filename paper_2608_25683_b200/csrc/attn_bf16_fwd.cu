@@ -231,23 +231,37 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
         f32x2 sum2 = make_f32x2(0.f, 0.f);
         const f32x2 neg_m2 = make_f32x2(-m, -m);
         float mx = -CUDART_INF_F;
+        // software pipeline over groups of 16 columns: the exp2 of group g+1 (MUFU pipe, 8 cycles per
+        // warp instruction) is issued before group g is summed, packed and stored
+        float e[2][16];
+        auto exps = [&](int g, float (&out)[16]) {
+          const int c = g >> 1, i0 = (g & 1) * 16;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int i = 0; i < 32; i += 2) {
+          for (int i = 0; i < 16; i += 2) {
             float a0, a1;
-            split_f32x2(fma2(make_f32x2(s[c][i], s[c][i + 1]), scale2, neg_m2), a0, a1);
-            float e0 = ex2(a0), e1 = ex2(a1);
-            if (masked) {
-              e0 = (c * 32 + i < limit) ? e0 : 0.f;
-              e1 = (c * 32 + i + 1 < limit) ? e1 : 0.f;
-            }
-            if (mx_out) mx = fmax3(mx, __uint_as_float(s[c][i]), __uint_as_float(s[c][i + 1]));
-            sum2 = add2(sum2, make_f32x2(e0, e1));
-            pk[i >> 1] = pack_bf16(e0, e1);
+            split_f32x2(fma2(make_f32x2(s[c][i0 + i], s[c][i0 + i + 1]), scale2, neg_m2), a0, a1);
+            out[i] = ex2(a0);
+            out[i + 1] = ex2(a1);
+            if (mx_out) mx = fmax3(mx, __uint_as_float(s[c][i0 + i]), __uint_as_float(s[c][i0 + i + 1]));
           }
-          tmem_st16(t_lane + c * 16, pk);
+        };
+        exps(0, e[0]);
+        uint32_t pk[16];
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          if (g + 1 < 8) exps(g + 1, e[(g + 1) & 1]);
+          float (&cur)[16] = e[g & 1];
+#pragma unroll
+          for (int i = 0; i < 16; i += 2) {
+            float e0 = cur[i], e1 = cur[i + 1];
+            if (masked) {
+              e0 = (g * 16 + i < limit) ? e0 : 0.f;
+              e1 = (g * 16 + i + 1 < limit) ? e1 : 0.f;
+            }
+            sum2 = add2(sum2, make_f32x2(e0, e1));
+            pk[(g & 1) * 8 + (i >> 1)] = pack_bf16(e0, e1);
+          }
+          if (g & 1) tmem_st16(t_lane + (g >> 1) * 16, pk);
         }
         if (mx_out) *mx_out = mx;
         float lo, hi;
