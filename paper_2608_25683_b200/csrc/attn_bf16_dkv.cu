@@ -517,13 +517,9 @@ psrl_status_t dkv_bf16(const AttnArgs& a) {
   }
   if (!ok) return PSRL_ERR_CUDA;
   const size_t smem = size_t(2 + 2 * ST) * kTileBytes + size_t(1 + 2 * ST) * kSliceBytes + 1024;
-  static bool attr_set = false;
-  cudaError_t e;
-  if (!attr_set) {
-    e = cudaFuncSetAttribute(dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return fail(e);
-    attr_set = true;
-  }
+  static bool attr_set[64] = {};
+  cudaError_t e = ensure_dynamic_smem(dkv_kernel, smem, attr_set);
+  if (e != cudaSuccess) return fail(e);
   Params p{};
   p.blob = P.dev;
   p.off_kvi = H.off_kvi; p.off_kvt = H.off_kvt; p.off_page_slot = H.off_page_slot; p.off_split = H.off_split;

@@ -320,13 +320,9 @@ psrl_status_t dq_bf16(const AttnArgs& a) {
             make_map_bf16_2d(&m.d_o, a.d_o, uint64_t(P.Hq) * 128, uint64_t(P.T_q), uint64_t(P.Hq) * 256, 128);
   if (!ok) return PSRL_ERR_CUDA;
   const size_t smem = size_t(2 + KS + VS) * kTileBytes + 1024;
-  static bool attr_set = false;
-  cudaError_t e;
-  if (!attr_set) {
-    e = cudaFuncSetAttribute(dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return fail(e);
-    attr_set = true;
-  }
+  static bool attr_set[64] = {};
+  cudaError_t e = ensure_dynamic_smem(dq_kernel, smem, attr_set);
+  if (e != cudaSuccess) return fail(e);
   Params p{};
   p.blob = P.dev;
   p.off_qt = H.off_qt; p.off_kvt = H.off_kvt; p.off_path_tiles = H.off_path_tiles;

@@ -411,11 +411,10 @@ psrl_status_t fwd_bf16(const AttnArgs& a) {
   p.part = a.part; p.part_lse = a.part_lse;
   p.status = a.status;
   const size_t smem = size_t(NQ + KS + VS) * kTileBytes + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+  static bool attr_set[64] = {};
+  {
+    const cudaError_t e = ensure_dynamic_smem(fwd_kernel, smem, attr_set);
     if (e != cudaSuccess) { set_last_cuda_error(e); return PSRL_ERR_CUDA; }
-    attr_set = true;
   }
   const int64_t grid = int64_t(P.q_tiles.size()) * P.Hkv * p.pairs_per_group;
   if (grid == 0) return PSRL_OK;

@@ -58,6 +58,19 @@ psrl_status_t merge_dq_bf16(const AttnArgs& a);   // dQ of those rows
 
 void set_last_cuda_error(cudaError_t e);
 
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute belongs to the
+// function on the current device; a process may drive several GPUs).
+template <class Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, size_t bytes, bool (&done)[64]) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes));
+  if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+  return e;
+}
+
 // Which backward kernels to launch (profiling aid): bit 0 delta, bit 1 dQ, bit 2 dK/dV.
 extern int g_bwd_phase_mask;
 
