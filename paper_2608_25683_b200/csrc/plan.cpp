@@ -399,7 +399,10 @@ psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out) {
       if (!P.seg_cascaded[a]) continue;
       const int32_t rows = P.seg_desc_q_end[a] - P.seg_desc_q_begin[a];
       const int32_t packed = (rows + kTile - 1) / kTile, nt = P.seg_n_kvt[a];
-      int64_t chunks = (kSms + packed * cta_units - 1) / (packed * cta_units);
+      // about half an SM count of forward CTAs for the packed part: the rows' own items need SMs too, and
+      // every further chunk adds a partial row per query row to merge (measured on the small-suffix case:
+      // 4 chunks 0.128 ms, 10 chunks 0.142 ms per step)
+      int64_t chunks = kSms / (2 * packed * cta_units);
       chunks = std::max<int64_t>(1, std::min<int64_t>(chunks, nt / 2));
       casc_part_base[a] = P.n_part_rows;
       casc_chunks[a] = static_cast<int32_t>(chunks);
