@@ -20,24 +20,33 @@ namespace {
 using namespace sm100;
 
 // ============================================================================ delta
+// 16 threads per (row, head): 16 bytes of O and of dO each, in memory order (a block reads 4 KB of each
+// tensor contiguously); D goes to its [Hq, T_q] layout.
 __global__ void __launch_bounds__(256)
 delta_kernel(int T_q, int Hq, const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
              float* __restrict__ delta) {
-  const int lane = threadIdx.x & 31;
-  const int64_t unit = int64_t(blockIdx.x) * 8 + (threadIdx.x >> 5);  // = h * T_q + r
-  if (unit >= int64_t(T_q) * Hq) return;
-  const int h = int(unit / T_q), r = int(unit % T_q);
-  const int64_t off = (int64_t(r) * Hq + h) * 128 + lane * 4;
-  const uint2 a = *reinterpret_cast<const uint2*>(o + off);
-  const uint2 b = *reinterpret_cast<const uint2*>(d_o + off);
-  const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.x));
-  const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&a.y));
-  const float2 b0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.x));
-  const float2 b1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b.y));
-  float s = a0.x * b0.x + a0.y * b0.y + a1.x * b1.x + a1.y * b1.y;
+  const int64_t i = int64_t(blockIdx.x) * 256 + threadIdx.x;   // 16-byte vector index
+  const int64_t unit = i >> 4;                                 // = r * Hq + h
+  const bool live = unit < int64_t(T_q) * Hq;
+  float s = 0.f;
+  if (live) {
+    const uint4 a = reinterpret_cast<const uint4*>(o)[i];
+    const uint4 b = reinterpret_cast<const uint4*>(d_o)[i];
+    const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-  for (int o2 = 16; o2 > 0; o2 >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o2);
-  if (lane == 0) delta[unit] = s;
+    for (int k = 0; k < 4; ++k) {
+      const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&av[k]));
+      const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&bv[k]));
+      s = fmaf(x.x, y.x, s);
+      s = fmaf(x.y, y.y, s);
+    }
+  }
+#pragma unroll
+  for (int o2 = 8; o2 > 0; o2 >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o2);
+  if (live && (threadIdx.x & 15) == 0) {
+    const int r = int(unit / Hq), h = int(unit % Hq);
+    delta[int64_t(h) * T_q + r] = s;
+  }
 }
 
 }  // namespace
@@ -49,7 +58,7 @@ psrl_status_t bwd_bf16(const AttnArgs& a) {
   if (P.T_q > 0 && (g_bwd_phase_mask & 1)) {
     // ---- D = rowsum(dO o O) ----
     const int64_t units = int64_t(P.T_q) * P.Hq;
-    delta_kernel<<<unsigned((units + 7) / 8), 256, 0, a.stream>>>(
+    delta_kernel<<<unsigned((units + 15) / 16), 256, 0, a.stream>>>(
         P.T_q, P.Hq, static_cast<const __nv_bfloat16*>(a.o), static_cast<const __nv_bfloat16*>(a.d_o), a.delta);
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
