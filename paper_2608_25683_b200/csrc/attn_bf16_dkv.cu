@@ -59,7 +59,9 @@ struct Params {
   int* status;
 };
 struct __align__(8) Barriers {
-  uint64_t kv_full, qd_full[ST], qd_empty[ST], s_full, dp_full, p_ready, ds_ready, acc_full;
+  // Q (+ the LSE slice) and dO (+ the D slice) of a step have barriers of their own: dO is free again after
+  // dV(i), Q only after dK(i), and the Q tile of the next step is what the tensor cores wait for
+  uint64_t kv_full, q_full[ST], q_empty[ST], do_full[ST], do_empty[ST], s_full, dp_full, p_ready, ds_ready, acc_full;
 };
 
 // The per-query-row terms of the backward are folded into the contractions as one extra
@@ -128,7 +130,10 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
   if (tid == 0) {
     s_abort = 0;
     mbar_init(&bar.kv_full, 1);
-    for (int i = 0; i < ST; ++i) { mbar_init(&bar.qd_full[i], 2); mbar_init(&bar.qd_empty[i], 1); }
+    for (int i = 0; i < ST; ++i) {
+      mbar_init(&bar.q_full[i], 2); mbar_init(&bar.q_empty[i], 1);
+      mbar_init(&bar.do_full[i], 2); mbar_init(&bar.do_empty[i], 1);
+    }
     mbar_init(&bar.s_full, 1); mbar_init(&bar.dp_full, 1);
     mbar_init(&bar.p_ready, 256); mbar_init(&bar.ds_ready, 256);
     mbar_init(&bar.acc_full, 1);
@@ -215,12 +220,18 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
         step(i, g, row0, nvq, diag, qpos0);
         const int h = hk * p.G + g;
         if (i + 1 < n_it) fetch(i + 1, lv_n, dv_n, nvq_next);
-        if (i >= ST) ok = mbar_wait(&bar.qd_empty[st], ((i / ST) + 1) & 1, abortp, p.status);
+        // dO's stage is released first (after dV of the step that used it), then Q's (after dK)
+        if (i >= ST) ok = mbar_wait(&bar.do_empty[st], ((i / ST) + 1) & 1, abortp, p.status);
         if (!ok) break;
         if (lane == 0) {
-          mbar_expect_tx(&bar.qd_full[st], 2 * kTileBytes);
-          load_row_tile(sQ + st * kTileBytes, &maps.q, &bar.qd_full[st], h, row0);
-          load_row_tile(sdO + st * kTileBytes, &maps.d_o, &bar.qd_full[st], h, row0);
+          mbar_expect_tx(&bar.do_full[st], kTileBytes);
+          load_row_tile(sdO + st * kTileBytes, &maps.d_o, &bar.do_full[st], h, row0);
+        }
+        if (i >= ST) ok = mbar_wait(&bar.q_empty[st], ((i / ST) + 1) & 1, abortp, p.status);
+        if (!ok) break;
+        if (lane == 0) {
+          mbar_expect_tx(&bar.q_full[st], kTileBytes);
+          load_row_tile(sQ + st * kTileBytes, &maps.q, &bar.q_full[st], h, row0);
         }
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
@@ -239,7 +250,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
         }
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bar.qd_full[st]);
+        if (lane == 0) { mbar_arrive(&bar.q_full[st]); mbar_arrive(&bar.do_full[st]); }
 #pragma unroll
         for (int x = 0; x < 4; ++x) { lv[x] = lv_n[x]; dv[x] = dv_n[x]; }
         nvq_cur = nvq_next;
@@ -281,7 +292,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       auto wait = [&](uint64_t* b, uint32_t parity) {
         return __all_sync(0xffffffffu, mbar_wait_relaxed(b, parity, abortp, p.status));
       };
-      bool ok = wait(&bar.kv_full, 0) && wait(&bar.qd_full[0], 0);
+      bool ok = wait(&bar.kv_full, 0) && wait(&bar.q_full[0], 0) && wait(&bar.do_full[0], 0);
       if (ok) {
         tc_fence_after();
         mma_kk(tmem + TM_ST, k_lo, q_lo, lsex_lo);
@@ -296,18 +307,21 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
         if (!ok) break;
         tc_fence_after();
         mma_acc(tmem + TM_DV, tmem + TM_ST, g_mn + so, i > 0);
+        commit(&bar.do_empty[i % ST]);          // dO(i) is done with: its stage may take dO(i + ST)
         if (i + 1 < n_it) {
-          // the Q / dO tiles of step i+1 arrive late (two-stage ring): wait behind dV(i), not before it
-          ok = wait(&bar.qd_full[(i + 1) % ST], ((i + 1) / ST) & 1);
+          // the Q tile of step i+1 arrives late (two-stage ring): wait behind dV(i), not before it
+          ok = wait(&bar.q_full[(i + 1) % ST], ((i + 1) / ST) & 1);
           if (!ok) break;
           mma_kk(tmem + TM_ST, k_lo, q_lo + so1, lsex_lo + sx1);
           commit(&bar.s_full);
         }
+        // dS^T(i) stored; in the same round, dO(i+1) (it landed long ago: its stage was released early)
         ok = wait(&bar.ds_ready, i & 1);
+        if (ok && i + 1 < n_it) ok = wait(&bar.do_full[(i + 1) % ST], ((i + 1) / ST) & 1);
         if (!ok) break;
         tc_fence_after();
         mma_acc(tmem + TM_DK, tmem + TM_DPT, q_mn + so, i > 0);
-        commit(&bar.qd_empty[i % ST]);
+        commit(&bar.q_empty[i % ST]);
         if (i + 1 < n_it) {
           mma_kk(tmem + TM_DPT, v_lo, g_lo + so1, dlx_lo + sx1);
           commit(&bar.dp_full);
