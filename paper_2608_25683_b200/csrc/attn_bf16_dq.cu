@@ -54,7 +54,7 @@ struct Params {
 };
 struct __align__(8) Barriers {
   uint64_t qdo_full, k_full[KS], k_empty[KS], v_full[VS], v_empty[VS];
-  uint64_t s_full, s_free, dp_full[2], ds_ready[2], dq_done;
+  uint64_t s_free, dp_full[2], ds_ready[2], dq_done;
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -80,7 +80,7 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     mbar_init(&bar.qdo_full, 1);
     for (int i = 0; i < KS; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1); }
     for (int i = 0; i < VS; ++i) { mbar_init(&bar.v_full[i], 1); mbar_init(&bar.v_empty[i], 1); }
-    mbar_init(&bar.s_full, 1); mbar_init(&bar.s_free, kSW * 32);
+    mbar_init(&bar.s_free, kSW * 32);
     for (int i = 0; i < 2; ++i) { mbar_init(&bar.dp_full[i], 1); mbar_init(&bar.ds_ready[i], kSW * 32); }
     mbar_init(&bar.dq_done, 1);
     fence_mbar_init();
@@ -141,7 +141,6 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     if (ok) {
       tc_fence_after();
       mma_kk(tmem + TM_S, q_lo, k_lo);
-      commit(&bar.s_full);
       mma_kk(tmem + TM_DP, g_lo, v_lo);
       commit(&bar.dp_full[0]);
       commit(&bar.v_empty[0]);
@@ -156,7 +155,6 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
         if (!ok) break;
         tc_fence_after();
         mma_kk(tmem + TM_S, q_lo, k_lo + ((j + 1) % KS) * (kTileBytes >> 4));
-        commit(&bar.s_full);
         mma_kk(tmem + TM_DP + ((j + 1) & 1) * 128, g_lo, v_lo + vs * (kTileBytes >> 4));
         commit(&bar.dp_full[(j + 1) & 1]);
         commit(&bar.v_empty[vs]);
@@ -197,10 +195,12 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       const int limit = diag ? min(row + 1, n_valid) : n_valid;   // keys [0, limit) are visible
       const bool need_mask = diag || n_valid < 128;
       // S(j) and dP(j) are both complete well before the warps get here (the MMA warp issues them
-      // one step ahead).  The whole score row goes to registers at once, so S may be overwritten.
+      // one step ahead).  One wait covers both: dP(j) is issued right behind S(j) by the same thread,
+      // and its commit tracks every MMA issued before it (a second wait would cost another
+      // shared-memory round trip of ~150 cycles per step, on the warps that set the pace).
+      // The whole score row goes to registers at once, so S may be overwritten.
       const uint32_t t_dp = t_lane + TM_DP + (j & 1) * 128;
-      ok = mbar_wait(&bar.s_full, j & 1, abortp, p.status) &&
-           mbar_wait(&bar.dp_full[j & 1], (j >> 1) & 1, abortp, p.status);
+      ok = mbar_wait(&bar.dp_full[j & 1], (j >> 1) & 1, abortp, p.status);
       if (!ok) break;
       tc_fence_after();
       uint32_t s[4][32], dp[2][32];

@@ -117,20 +117,39 @@ __device__ __forceinline__ bool mbar_test_relaxed(uint64_t* bar, uint32_t parity
   return ok != 0;
 }
 
+// Non-blocking test of three phases in one shared-memory round trip: the three test_wait
+// instructions are independent and issue back to back; only the final combination waits for them.
+__device__ __forceinline__ bool mbar_test3_relaxed(uint64_t* b0, uint32_t p0, uint64_t* b1, uint32_t p1, uint64_t* b2,
+                                                   uint32_t p2) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p, q, r;\n\t"
+      "mbarrier.test_wait.parity.relaxed.cta.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.test_wait.parity.relaxed.cta.shared::cta.b64 q, [%3], %4;\n\t"
+      "mbarrier.test_wait.parity.relaxed.cta.shared::cta.b64 r, [%5], %6;\n\t"
+      "and.pred p, p, q;\n\t"
+      "and.pred p, p, r;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(b0)), "r"(p0), "r"(smem_u32(b1)), "r"(p1), "r"(smem_u32(b2)), "r"(p2)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait of the MMA-issuing warp on up to three barriers at once.  A wait costs that warp
 // 100-350 cycles even when the phase is already complete (the barrier lives in shared memory,
 // whose pipeline the running MMAs keep busy, and the warp competes with the softmax warps for
 // issue slots), and the tensor pipe queues only a few MMAs, so every separate wait between two
-// groups of MMAs opens a bubble.  The first barrier is the one expected to complete last: the warp
-// blocks on it with try_wait (suspended by the hardware, no issue slots taken from the softmax
-// warps), then tests the other two side by side.  All lanes take part (warp-uniform result).
+// groups of MMAs opens a bubble.  Usually all three phases are complete when the warp gets here:
+// one combined test (a single round trip) then suffices.  Otherwise the warp blocks on the first
+// barrier, the one expected to complete last, with try_wait (suspended by the hardware, no issue
+// slots taken from the softmax warps) and tests again.  All lanes take part (warp-uniform result).
 __device__ __forceinline__ bool mbar_wait_all3(uint64_t* b0, uint32_t p0, uint64_t* b1, uint32_t p1, uint64_t* b2,
                                                uint32_t p2, volatile int* s_abort, int* g_status) {
+  if (__all_sync(0xffffffffu, mbar_test3_relaxed(b0, p0, b1, p1, b2, p2))) return true;
   if (!__all_sync(0xffffffffu, mbar_wait_relaxed(b0, p0, s_abort, g_status))) return false;
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    const bool t1 = mbar_test_relaxed(b1, p1);
-    const bool t2 = mbar_test_relaxed(b2, p2);
-    if (__all_sync(0xffffffffu, t1 && t2)) return true;
+    if (__all_sync(0xffffffffu, mbar_test3_relaxed(b0, p0, b1, p1, b2, p2))) return true;
     if (it > 1024 && *s_abort) return false;
   }
   *s_abort = 1;
