@@ -337,6 +337,53 @@ def flat_runner(lib, r, device, head_slice=None):
     return Runner(lib, fw, 0, device, data=(q, k, v, d_o))
 
 
+def library_context_leg(lib, w, V, device, ms_tree, flops, iters):
+    """Context, not a target and not the oracle: a library's varlen causal attention (flash_attn's
+    kernels as shipped in the image) forward + backward on the flattened, unshared layout: every
+    sample a sequence of its own.  Timing does not depend on the values, so inputs are random."""
+    import torch
+    try:
+        import flash_attn
+        from flash_attn import flash_attn_varlen_func
+    except Exception as ex:
+        return {"unavailable": str(ex)[:120]}
+    _, lens, _, _, _ = lib.flatten_forest(V)
+    lens = [int(x) for x in lens]
+    Hq, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
+    T = sum(lens)
+    # Slices of heads keep every tensor below 2^31 elements: on c4's unshared layout (4.3e9 elements per
+    # Q-shaped tensor) the library raised an illegal memory access, so it is never handed such a tensor.
+    hq, hkv = Hq, Hkv
+    if T * hq * d >= 2 ** 31 or T * Hq * d * 2 * 4 >= 60e9:
+        hq, hkv = Hq // Hkv, 1
+    while T * hq * d >= 2 ** 31 and hq > 1:
+        hq //= 2
+    if T * hq * d >= 2 ** 31:
+        return {"skipped": "a single head of the unshared layout exceeds 2^31 elements"}
+    slices = Hq // hq
+    try:
+        cu = torch.tensor(np.concatenate([[0], np.cumsum(lens)]), dtype=torch.int32, device=device)
+        q = torch.randn(T, hq, d, device=device, dtype=torch.bfloat16, requires_grad=True)
+        k = torch.randn(T, hkv, d, device=device, dtype=torch.bfloat16, requires_grad=True)
+        v = torch.randn(T, hkv, d, device=device, dtype=torch.bfloat16, requires_grad=True)
+        d_o = torch.randn(T, hq, d, device=device, dtype=torch.bfloat16)
+
+        def step():
+            o = flash_attn_varlen_func(q, k, v, cu, cu, max(lens), max(lens), softmax_scale=w.softmax_scale, causal=True)
+            o.backward(d_o)
+            q.grad = k.grad = v.grad = None
+
+        ms = time_region(step, iters, 2) * slices
+    except Exception as ex:
+        return {"library": "flash_attn " + flash_attn.__version__, "error": str(ex)[:200]}
+    flat_flops = dedup_flops(d, Hq, V["flat_pairs"])
+    return {"library": "flash_attn " + flash_attn.__version__ + " flash_attn_varlen_func, causal, fwd + autograd bwd",
+            "layout": "flattened unshared: %d sequences, %d tokens" % (len(lens), T), "kv_head_slices": slices,
+            "ms_per_step": round(ms, 3), "tflops_on_unshared_flops": round(flat_flops / (ms * 1e-3) / 1e12, 1),
+            "dedup_tflops_equivalent": round(flops / (ms * 1e-3) / 1e12, 1),
+            "tree_path_speedup_over_library": round(ms / ms_tree, 2)}
+
+
 def forest_of_groups(w, groups):
     """The sub-forest of `w` made of the prefix groups `groups` (root indices counted in input order)."""
     from paper_2608_25683_b200.workloads import Workload
@@ -479,6 +526,8 @@ def main():
     ap.add_argument("--ref-samples", type=int, default=2, help="samples per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-unshared", action="store_true")
+    ap.add_argument("--context", action="store_true",
+                    help="also time a library's varlen attention (flash_attn) on the unshared layout, for context")
     ap.add_argument("--block-size", default=None,
                     help="override the page size of every group: 16|32|64|128|256, or 'adaptive' (one extent per span)")
     ap.add_argument("--length-scale", type=float, default=1.0,
@@ -516,6 +565,15 @@ def main():
         bs = 0 if args.block_size == "adaptive" else int(args.block_size)
         w.group_block_size = [bs] * len(w.group_block_size)
         w.free_extents = None
+    t0 = time.perf_counter()
+    _p = lib.Plan(w.parent, w.seg_len, w.group_block_size, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype,
+                  w.seg_flags, w.free_extents)
+    t1 = time.perf_counter()
+    _p.upload(device)
+    torch.cuda.synchronize()
+    plan_ms = {"build_ms": round((t1 - t0) * 1e3, 3), "upload_ms": round((time.perf_counter() - t1) * 1e3, 3),
+               "device_bytes": _p.device_bytes()}
+    del _p
     r = Runner(lib, w, dist_util.rank_seed(args.seed, rank) + 1, device)
     V = r.plan.view
     flops = dedup_flops(w.head_dim, w.n_q_heads, V["tree_pairs"])
@@ -565,6 +623,31 @@ def main():
             dist.barrier()
             dist.destroy_process_group()
         return
+
+    # ---- every step on its own (median, min) and bitwise reproducibility over three runs ----
+    n_each = max(5, min(args.steps, 20))
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_each + 1)]
+    if flush is None:
+        evs[0].record()
+        for i in range(n_each):
+            r.step()
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        each = [evs[i].elapsed_time(evs[i + 1]) for i in range(n_each)]
+    else:
+        each = [time_region(r.step, 1, 0, flush) for _ in range(n_each)]
+    step_stats = {"n": n_each, "median_ms": round(float(np.median(each)), 4), "min_ms": round(min(each), 4),
+                  "max_ms": round(max(each), 4)}
+    outs = (r.o, r.lse, r.dq, r.dk, r.dv)
+    first = [x.clone() for x in outs]
+    same = True
+    for _ in range(2):
+        r.step()
+        same = same and all(torch.equal(a.view(torch.int16 if a.element_size() == 2 else torch.int32),
+                                        b.view(torch.int16 if b.element_size() == 2 else torch.int32))
+                            for a, b in zip(first, outs))
+    del first
+    torch.cuda.empty_cache()
 
     pk = peaks()
     # ---- per-kernel times (each kernel alone, CUDA events on the launch stream) ----
@@ -626,6 +709,7 @@ def main():
            "h2d_bytes_per_step": nbytes(hq, hk, hv, hdo), "d2h_bytes_per_step": nbytes(ho, hl, hdq, hdk, hdv)}
 
     # ---- the same kernels on the unshared (flattened) layout ----
+    print("[bench] tree path measured; unshared leg", file=sys.stderr, flush=True)
     unshared = None
     if not args.no_unshared and world == 1:
         try:
@@ -642,6 +726,15 @@ def main():
                         "kv_head_slices": slices}
         except Exception as ex:  # e.g. out of memory on the flattened tensors
             unshared = {"error": str(ex)[:200]}
+
+    context = None
+    if args.context and world == 1:
+        torch.cuda.synchronize()
+        print("[bench] library context leg", file=sys.stderr, flush=True)
+        context = library_context_leg(lib, w, V, device, ms, flops, max(3, min(args.steps, 10)))
+        torch.cuda.synchronize()
+        print("[bench] library context leg done", file=sys.stderr, flush=True)
+        torch.cuda.empty_cache()
 
     pack = None
     if args.pack and world == 1:
@@ -677,7 +770,8 @@ def main():
                     "per-step working set exceeds the 126 MB L2 (inputs larger than L2); no explicit flush" if flush is None
                     else "working set fits in the L2: a 252 MB buffer is overwritten before every timed step "
                          "(each step timed on its own, flush outside the timed part)")), clocks=clocks.summary(), e2e=e2e, gpu_launches=(lib.psrl_launch_count(r.plan, False) + lib.psrl_launch_count(r.plan, True)) * args.steps,
-                roofline=roofline, cpu_baseline=cpu, unshared=unshared, microbatch=micro, schedule=sched, kv_pack=pack,
+                roofline=roofline, cpu_baseline=cpu, step_ms=step_stats, bitwise_reproducible_3_runs=bool(same),
+                plan=plan_ms, unshared=unshared, library_context=context, microbatch=micro, schedule=sched, kv_pack=pack,
                 frac_of_bf16_peak={"burst": round(value / world / pk["bf16_tflops"], 4),
                                    "sustained": round(value / world / pk["bf16_tflops_sustained"], 4)})
     print(json.dumps(line), flush=True)
