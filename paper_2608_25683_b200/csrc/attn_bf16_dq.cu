@@ -32,6 +32,7 @@ namespace {
 using namespace sm100;
 
 constexpr int KS = 3, VS = 2;                 // K and V ring depths
+constexpr int kPolyPerGroup = 4;                 // of every 16 exponentials, this many are computed on the FMA pipes
 constexpr int kSW = 4;                        // softmax-backward warps: one per SM sub-partition
 constexpr int kThreads = (kSW + 2) * 32;
 constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 384;   // dP / dS is double-buffered: 128 and 256
@@ -51,6 +52,8 @@ struct Params {
   __nv_bfloat16* d_q;
   float* part;  // unscaled fp32 dQ rows [n_part_rows][Hq][128] of items that do not own their rows
   int* status;
+  int* done_ctr;   // CTAs whose producers have issued their last load
+  int32_t resident;  // CTAs resident at once (one per SM)
 };
 struct __align__(8) Barriers {
   uint64_t qdo_full, k_full[KS], k_empty[KS], v_full[VS], v_empty[VS];
@@ -113,6 +116,16 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
         if (j >= VS && !mbar_wait_sleepy(&bar.v_empty[vs], ((j / VS) + 1) & 1, abortp, p.status)) break;
         load_kv_tile_at(sV + vs * kTileBytes, maps.kv.v, &bar.v_full[vs], cur, head_row0);
         cur = nxt;
+      }
+      // The k-th CTA to get this far is about to make room for CTA `resident + k` (CTAs start in index
+      // order, one per SM): its Q and dO tiles go to the L2 now, so that its first step does not wait for HBM.
+      const int nb = atomicAdd(p.done_ctr, 1) + p.resident;
+      if (nb < int(gridDim.x)) {
+        const int nrow = reinterpret_cast<const QTile*>(p.blob + p.off_qt)[nb / p.Hq].q_row0, nh = nb % p.Hq;
+        tma_prefetch_2d(&maps.q, nh * 128, nrow);
+        tma_prefetch_2d(&maps.q, nh * 128 + 64, nrow);
+        tma_prefetch_2d(&maps.d_o, nh * 128, nrow);
+        tma_prefetch_2d(&maps.d_o, nh * 128 + 64, nrow);
       }
     }
   } else if (warp == kSW + 1) {
@@ -227,10 +240,15 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
           const int c = half * 2 + (g >> 1), i0 = (g & 1) * 16;
 #pragma unroll
           for (int i = 0; i < 16; i += 2) {
-            float a0, a1;
-            split_f32x2(fma2(make_f32x2(s[c][i0 + i], s[c][i0 + i + 1]), scale2, neg_lse2), a0, a1);
-            out[i] = ex2(a0);
-            out[i + 1] = ex2(a1);
+            const f32x2 a = fma2(make_f32x2(s[c][i0 + i], s[c][i0 + i + 1]), scale2, neg_lse2);
+            if (i < kPolyPerGroup) {   // a share of the exponentials goes to the FMA pipes
+              ex2_fma_pair(a, out[i], out[i + 1]);
+            } else {
+              float a0, a1;
+              split_f32x2(a, a0, a1);
+              out[i] = ex2(a0);
+              out[i + 1] = ex2(a1);
+            }
           }
         };
         exps(0, pe[0]);
@@ -270,21 +288,17 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
     if (ok) ok = mbar_wait(&bar.dq_done, 0, abortp, p.status);
     if (ok) {
       tc_fence_after();
-      __nv_bfloat16* drow = p.d_q + (int64_t(qt.q_row0 + row) * p.Hq + h) * 128;
+      // Final rows leave through shared memory (the K ring is idle by now: every MMA has completed), so
+      // that a warp's store instruction covers two whole 256-byte rows instead of 16 bytes of 32 rows.
+      // A warp stages only its own 32 rows: 272-byte pitch, no bank conflicts either way, no CTA barrier.
+      constexpr int kPitch = 272;
+      uint8_t* stage = sK + warp * (32 * kPitch);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t r[32];
         tmem_ld32(t_lane + TM_DQ + c * 32, r);
         tmem_wait_ld();
-        if (row_ok && qt.part_row0 >= 0) {
-          // the row has other contributors: unscaled fp32 partial, summed by the merge kernel
-          float* prow = p.part + (int64_t(qt.part_row0 + row) * p.Hq + h) * 128 + c * 32;
-#pragma unroll
-          for (int x = 0; x < 8; ++x)
-            *reinterpret_cast<float4*>(prow + x * 4) =
-                make_float4(__uint_as_float(r[4 * x]), __uint_as_float(r[4 * x + 1]), __uint_as_float(r[4 * x + 2]),
-                            __uint_as_float(r[4 * x + 3]));
-        } else if (row_ok) {
+        if (qt.part_row0 < 0) {
 #pragma unroll
           for (int x = 0; x < 4; ++x) {
             uint4 v;
@@ -292,8 +306,29 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
             v.y = pack_bf16(__uint_as_float(r[8 * x + 2]) * p.scale, __uint_as_float(r[8 * x + 3]) * p.scale);
             v.z = pack_bf16(__uint_as_float(r[8 * x + 4]) * p.scale, __uint_as_float(r[8 * x + 5]) * p.scale);
             v.w = pack_bf16(__uint_as_float(r[8 * x + 6]) * p.scale, __uint_as_float(r[8 * x + 7]) * p.scale);
-            *reinterpret_cast<uint4*>(drow + c * 32 + x * 8) = v;
+            *reinterpret_cast<uint4*>(stage + lane * kPitch + c * 64 + x * 16) = v;
           }
+          continue;
+        }
+        if (row_ok) {
+          // the row has other contributors: unscaled fp32 partial, summed by the merge kernel
+          float* prow = p.part + (int64_t(qt.part_row0 + row) * p.Hq + h) * 128 + c * 32;
+#pragma unroll
+          for (int x = 0; x < 8; ++x)
+            *reinterpret_cast<float4*>(prow + x * 4) =
+                make_float4(__uint_as_float(r[4 * x]), __uint_as_float(r[4 * x + 1]), __uint_as_float(r[4 * x + 2]),
+                            __uint_as_float(r[4 * x + 3]));
+        }
+      }
+      if (qt.part_row0 < 0) {
+        __syncwarp();
+        const int sub = lane >> 4, piece = lane & 15;
+#pragma unroll 4
+        for (int it = 0; it < 16; ++it) {
+          const int rr = it * 2 + sub;                      // row inside the warp's 32
+          const uint4 v = *reinterpret_cast<const uint4*>(stage + rr * kPitch + piece * 16);
+          if (warp * 32 + rr < qt.n_rows)
+            *reinterpret_cast<uint4*>(p.d_q + (int64_t(qt.q_row0 + warp * 32 + rr) * p.Hq + h) * 128 + piece * 8) = v;
         }
       }
     }
@@ -331,6 +366,7 @@ psrl_status_t dq_bf16(const AttnArgs& a) {
   p.cap = cap; p.scale = a.scale; p.scale_log2 = a.scale * kLog2e;
   p.lse = a.lse_in; p.delta = a.delta; p.d_q = static_cast<__nv_bfloat16*>(a.d_q); p.status = a.status;
   p.part = a.part;
+  p.done_ctr = a.status + kWsCtrDq; p.resident = resident_ctas();
   const int64_t grid = int64_t(P.q_tiles.size()) * P.Hq;
   if (grid > INT32_MAX) return PSRL_ERR_SHAPE;
   dq_kernel<<<unsigned(grid), kThreads, smem, a.stream>>>(m, p);

@@ -10,6 +10,11 @@ namespace psrl {
 //   forward:  partial O rows, their LSE
 //   backward: D = rowsum(dO o O) as fp32 [Hq, T_q], partial dV/dK slabs, partial dQ rows.
 constexpr size_t kWsHeaderBytes = 256;
+// Control words 16..18: per-kernel counters of CTAs whose producers have issued their last load
+// (forward, dQ, dK/dV); zeroed with the header before every call.
+constexpr int kWsCtrFwd = 16, kWsCtrDq = 17, kWsCtrDkv = 18;
+// CTAs of a one-CTA-per-SM kernel that are resident at once (the device's SM count).
+int resident_ctas();
 // After D: fp32 partial dV/dK slabs of split KV tiles, [slab][kv head][dV, dK][128][128].
 constexpr size_t kSlabBytes = size_t(2) * 128 * 128 * sizeof(float);
 inline size_t ws_delta_bytes(const Plan& P) {

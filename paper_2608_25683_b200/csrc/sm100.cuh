@@ -194,6 +194,13 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
+// L2 prefetch of one box of a tiled tensor map (no shared-memory destination, no barrier).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* m, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(m)),
+               "r"(x), "r"(y)
+               : "memory");
+}
+
 // ---------------------------------------------------------------- tensor memory
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
@@ -365,6 +372,41 @@ __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
   f32x2 r;
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
   return r;
+}
+
+__device__ __forceinline__ f32x2 add2_rm(f32x2 a, f32x2 b) {   // rounded towards minus infinity
+  f32x2 r;
+  asm("add.rm.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+  return r;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+  return r;
+}
+
+// 2^x for a pair of arguments on the FMA pipes instead of the MUFU (whose 4 results per cycle and
+// sub-partition bound the softmax warps): x = n + f with n = floor(x) from an add of 1.5 * 2^23
+// rounded down (n sits in the low mantissa bits of the sum), 2^f on [0, 1) by a cubic fitted for the
+// smallest maximal relative error (8.6e-5, far below bf16's 2^-9), and n added into the exponent
+// field.  Arguments are clamped at -126 (results below 2^-126 come out as ~2^-126 instead of 0:
+// both vanish in bf16 products of this kernel's magnitudes); arguments above ~127 are not supported.
+__device__ __forceinline__ void ex2_fma_pair(f32x2 x, float& r0, float& r1) {
+  float x0, x1;
+  split_f32x2(x, x0, x1);
+  const f32x2 xc = make_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const f32x2 magic = make_f32x2(12582912.f, 12582912.f);
+  const f32x2 t = add2_rm(xc, magic);
+  const f32x2 f = sub2(xc, sub2(t, magic));
+  const f32x2 c1 = make_f32x2(0.6951167583465576f, 0.6951167583465576f),
+              c2 = make_f32x2(0.22764499485492706f, 0.22764499485492706f),
+              c3 = make_f32x2(0.07706703990697861f, 0.07706703990697861f), one = make_f32x2(1.f, 1.f);
+  const f32x2 pl = fma2(fma2(fma2(c3, f, c2), f, c1), f, one);
+  float p0, p1, t0, t1;
+  split_f32x2(pl, p0, p1);
+  split_f32x2(t, t0, t1);
+  r0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
+  r1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
 }
 
 // max of three in one instruction
