@@ -56,6 +56,8 @@ struct FwdParams {
   float* part;      // partial rows [n_part_rows][Hq][128]: normalised O of items that do not own their rows
   float* part_lse;  // [n_part_rows][Hq]
   int* status;
+  int* done_ctr;     // CTAs whose producers have issued their last load
+  int32_t resident;  // CTAs resident at once (one per SM)
 };
 
 struct __align__(8) Barriers {
@@ -127,6 +129,18 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
         if (j >= VS && !mbar_wait_sleepy(&bar.v_empty[vs], ((j / VS) + 1) & 1, abortp, p.status)) break;
         load_kv_tile_at(sV + vs * kTileBytes, maps.kv.v, &bar.v_full[vs], cur, head_row0);
         cur = nxt;
+      }
+      // The k-th CTA to get this far is about to make room for CTA `resident + k` (CTAs start in index
+      // order, one per SM): its Q tiles go to the L2 now, so that its first step does not wait for HBM.
+      const int nb = atomicAdd(p.done_ctr, 1) + p.resident;
+      if (nb < int(gridDim.x)) {
+        const int nu = nb % units, npair = nu % p.pairs_per_group;
+        const int nh0 = (nu / p.pairs_per_group) * p.G + npair * NQ, nnq = min(NQ, p.G - npair * NQ);
+        const int nrow = reinterpret_cast<const QTile*>(p.blob + p.off_qt)[nb / units].q_row0;
+        for (int q = 0; q < nnq; ++q) {
+          tma_prefetch_2d(&maps.q, (nh0 + q) * 128, nrow);
+          tma_prefetch_2d(&maps.q, (nh0 + q) * 128 + 64, nrow);
+        }
       }
     }
   } else if (warp == 4 * NQ + 1) {
@@ -338,7 +352,12 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       const bool store = row < qt.n_rows;
       const int h = h0 + q;
       const bool partial = qt.part_row0 >= 0;
-      __nv_bfloat16* orow = p.o + (int64_t(qt.q_row0 + row) * p.Hq + h) * 128;
+      // Final rows leave through shared memory (the Q tiles and the K ring are idle by now: every
+      // S = Q K^T has completed), so that a warp's store instruction covers two whole 256-byte rows
+      // instead of 16 bytes of 32 rows.  A warp stages only its own 32 rows: 272-byte pitch, no bank
+      // conflicts either way, no CTA barrier.
+      constexpr int kPitch = 272;
+      uint8_t* stage = sQ + warp * (32 * kPitch);
       float* prow = p.part + (int64_t(qt.part_row0 + row) * p.Hq + h) * 128;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
@@ -359,10 +378,20 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
 #pragma unroll
         for (int i = 0; i < 32; i += 2)
           pk[i >> 1] = pack_bf16(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
-        if (store) {
 #pragma unroll
-          for (int x = 0; x < 4; ++x)
-            *reinterpret_cast<uint4*>(orow + c * 32 + x * 8) = make_uint4(pk[4 * x], pk[4 * x + 1], pk[4 * x + 2], pk[4 * x + 3]);
+        for (int x = 0; x < 4; ++x)
+          *reinterpret_cast<uint4*>(stage + lane * kPitch + c * 64 + x * 16) =
+              make_uint4(pk[4 * x], pk[4 * x + 1], pk[4 * x + 2], pk[4 * x + 3]);
+      }
+      if (!partial) {
+        __syncwarp();
+        const int sub = lane >> 4, piece = lane & 15, wrow0 = (warp & 3) * 32;
+#pragma unroll 4
+        for (int it = 0; it < 16; ++it) {
+          const int rr = it * 2 + sub;                      // row inside the warp's 32
+          const uint4 v = *reinterpret_cast<const uint4*>(stage + rr * kPitch + piece * 16);
+          if (wrow0 + rr < qt.n_rows)
+            *reinterpret_cast<uint4*>(p.o + (int64_t(qt.q_row0 + wrow0 + rr) * p.Hq + h) * 128 + piece * 8) = v;
         }
       }
       if (store && partial) p.part_lse[int64_t(qt.part_row0 + row) * p.Hq + h] = (m_ref + log2f(l_run)) * kLn2;
@@ -410,6 +439,7 @@ psrl_status_t fwd_bf16(const AttnArgs& a) {
   p.lse = a.lse_out;
   p.part = a.part; p.part_lse = a.part_lse;
   p.status = a.status;
+  p.done_ctr = a.status + kWsCtrFwd; p.resident = resident_ctas();
   const size_t smem = size_t(NQ + KS + VS) * kTileBytes + 1024;
   static bool attr_set[64] = {};
   {
