@@ -702,11 +702,62 @@ def main():
         ho.copy_(r.o, non_blocking=True); hl.copy_(r.lse, non_blocking=True); hdq.copy_(r.dq, non_blocking=True)
         hdk.copy_(r.dk, non_blocking=True); hdv.copy_(r.dv, non_blocking=True)
 
-    e2e_ms = time_region(e2e_step, max(3, min(args.steps, 10)), 2)
+    n_e2e = max(4, min(args.steps, 10))
+    e2e_serial_ms = time_region(e2e_step, n_e2e, 2)
+
+    # The same, software-pipelined the way a training loop feeds a device: three streams and two sets of device
+    # buffers, so that step i+1's host->device copies and step i-1's device->host copies run beside step i.
+    # Every step still copies all its inputs in and all its outputs out inside the timed region.
+    r2 = Runner(lib, w, 0, device, data=tuple(x.clone() for x in (r.q, r.k, r.v, r.d_o)))
+    pair = (r, r2)
+    s_in, s_c, s_out = (torch.cuda.Stream(device=device) for _ in range(3))
+
+    def e2e_pipelined(n):
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_c = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
+        cur = torch.cuda.current_stream()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(cur)
+        for st in (s_in, s_c, s_out):
+            st.wait_event(t0)
+        for i in range(n):
+            b = i & 1
+            x = pair[b]
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_c[b])        # the inputs of set b are free once step i-2 has run
+                x.q.copy_(hq, non_blocking=True); x.k.copy_(hk, non_blocking=True)
+                x.v.copy_(hv, non_blocking=True); x.d_o.copy_(hdo, non_blocking=True)
+                ev_in[b].record(s_in)
+            with torch.cuda.stream(s_c):
+                s_c.wait_event(ev_in[b])
+                if i >= 2:
+                    s_c.wait_event(ev_out[b])       # the outputs of set b have been read back
+                x.step()
+                ev_c[b].record(s_c)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_c[b])
+                ho.copy_(x.o, non_blocking=True); hl.copy_(x.lse, non_blocking=True); hdq.copy_(x.dq, non_blocking=True)
+                hdk.copy_(x.dk, non_blocking=True); hdv.copy_(x.dv, non_blocking=True)
+                ev_out[b].record(s_out)
+        for st in (s_in, s_c, s_out):
+            cur.wait_stream(st)
+        t1.record(cur)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / n
+
+    e2e_pipelined(2)
+    e2e_ms = e2e_pipelined(n_e2e)
+    del r2, pair
+    torch.cuda.empty_cache()
     es = 2 if w.dtype == "bf16" else 4
     nbytes = lambda *ts: int(sum(x.numel() * x.element_size() for x in ts))
     e2e = {"value": round(flops / (e2e_ms * 1e-3) / 1e12 * world, 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
-           "h2d_bytes_per_step": nbytes(hq, hk, hv, hdo), "d2h_bytes_per_step": nbytes(ho, hl, hdq, hdk, hdv)}
+           "h2d_bytes_per_step": nbytes(hq, hk, hv, hdo), "d2h_bytes_per_step": nbytes(ho, hl, hdq, hdk, hdv),
+           "mode": "three streams, two sets of device buffers: copies of neighbouring steps overlap the kernels",
+           "serial": {"value": round(flops / (e2e_serial_ms * 1e-3) / 1e12 * world, 3),
+                      "ms_per_step": round(e2e_serial_ms, 3), "mode": "copy in, run, copy out on one stream"}}
 
     # ---- the same kernels on the unshared (flattened) layout ----
     print("[bench] tree path measured; unshared leg", file=sys.stderr, flush=True)
