@@ -41,6 +41,8 @@ constexpr int ST = 2;                              // (Q, dO) tile ring depth
 static_assert(kSubRows == 128, "the dK/dV kernel steps through 128-row query tiles");
 constexpr int kThreads = (8 + 2) * 32;             // 8 softmax-backward warps + producer + MMA
 constexpr uint32_t TM_ST = 0, TM_DPT = 128, TM_DV = 256, TM_DK = 384;
+// named barriers (softmax warps arrive, the MMA warp syncs): P^T(i) stored, dS^T(i) stored
+constexpr uint32_t kBarP = 1, kBarDs = 2, kBarThreads = 8 * 32 + 32;
 
 struct Maps {
   CUtensorMap q, d_o;  // boxes of 128 rows x 64 columns
@@ -61,7 +63,7 @@ struct Params {
 struct __align__(8) Barriers {
   // Q (+ the LSE slice) and dO (+ the D slice) of a step have barriers of their own: dO is free again after
   // dV(i), Q only after dK(i), and the Q tile of the next step is what the tensor cores wait for
-  uint64_t kv_full, q_full[ST], q_empty[ST], do_full[ST], do_empty[ST], s_full, dp_full, p_ready, ds_ready, acc_full;
+  uint64_t kv_full, q_full[ST], q_empty[ST], do_full[ST], do_empty[ST], s_full, dp_full, acc_full;
 };
 
 // The per-query-row terms of the backward are folded into the contractions as one extra
@@ -135,7 +137,6 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       mbar_init(&bar.do_full[i], 2); mbar_init(&bar.do_empty[i], 1);
     }
     mbar_init(&bar.s_full, 1); mbar_init(&bar.dp_full, 1);
-    mbar_init(&bar.p_ready, 256); mbar_init(&bar.ds_ready, 256);
     mbar_init(&bar.acc_full, 1);
     fence_mbar_init();
   }
@@ -303,8 +304,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       for (int i = 0; ok && i < n_it; ++i) {
         const uint32_t so = (i % ST) * (kTileBytes >> 4), so1 = ((i + 1) % ST) * (kTileBytes >> 4);
         const uint32_t sx1 = ((i + 1) % ST) * (kSliceBytes >> 4);
-        ok = wait(&bar.p_ready, i & 1);
-        if (!ok) break;
+        named_sync(kBarP, kBarThreads);
         tc_fence_after();
         mma_acc(tmem + TM_DV, tmem + TM_ST, g_mn + so, i > 0);
         commit(&bar.do_empty[i % ST]);          // dO(i) is done with: its stage may take dO(i + ST)
@@ -316,8 +316,8 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
           commit(&bar.s_full);
         }
         // dS^T(i) stored; in the same round, dO(i+1) (it landed long ago: its stage was released early)
-        ok = wait(&bar.ds_ready, i & 1);
-        if (ok && i + 1 < n_it) ok = wait(&bar.do_full[(i + 1) % ST], ((i + 1) / ST) & 1);
+        named_sync(kBarDs, kBarThreads);
+        if (i + 1 < n_it) ok = wait(&bar.do_full[(i + 1) % ST], ((i + 1) / ST) & 1);
         if (!ok) break;
         tc_fence_after();
         mma_acc(tmem + TM_DK, tmem + TM_DPT, q_mn + so, i > 0);
@@ -342,10 +342,11 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       float pr[64];  // this thread's P^T values, kept for the second half-step
       // ---- half-step 1: P^T = exp2(c S^T_aug); -LSE / scale is already inside S^T_aug, and
       //      a query row beyond the valid range carries -inf there, so its column comes out 0 ----
-      ok = mbar_wait(&bar.s_full, i & 1, abortp, p.status);
-      if (!ok) break;
-      tc_fence_after();
-      {
+      // (a warp that gave up on a wait still walks the loop and performs every arrival on the named
+      // barriers, so that the MMA warp is never left waiting at one)
+      if (ok) ok = mbar_wait(&bar.s_full, i & 1, abortp, p.status);
+      if (ok) {
+        tc_fence_after();
         uint32_t s[2][32];
         tmem_ld32(t_lane + TM_ST + wg * 64, s[0]);
         tmem_ld32(t_lane + TM_ST + wg * 64 + 32, s[1]);
@@ -384,12 +385,11 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       }
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bar.p_ready);
+      named_arrive(kBarP, kBarThreads);
       // ---- half-step 2: dS^T = P^T o dP^T_aug (-D is already inside) ----
-      ok = mbar_wait(&bar.dp_full, i & 1, abortp, p.status);
-      if (!ok) break;
-      tc_fence_after();
-      {
+      if (ok) ok = mbar_wait(&bar.dp_full, i & 1, abortp, p.status);
+      if (ok) {
+        tc_fence_after();
         uint32_t dp[2][32];
         tmem_ld32(t_lane + TM_DPT + wg * 64, dp[0]);
         tmem_ld32(t_lane + TM_DPT + wg * 64 + 32, dp[1]);
@@ -408,7 +408,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       }
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bar.ds_ready);
+      named_arrive(kBarDs, kBarThreads);
     }
     // ---- epilogue: warps 0-3 take dV, warps 4-7 take dK ----
     if (ok && n_it > 0) ok = mbar_wait(&bar.acc_full, 0, abortp, p.status);

@@ -39,6 +39,8 @@ using namespace sm100;
 constexpr int NQ = 2;                    // query heads per CTA
 constexpr int KS = 2, VS = 2;            // K and V ring depths
 constexpr int kThreads = (4 * NQ + 2) * 32;
+// named barriers (the softmax warps of head q arrive, the MMA warp syncs): P_q of a tile stored
+constexpr uint32_t kBarP = 1, kBarThreads = 128 + 32;
 
 struct FwdMaps {
   CUtensorMap q;
@@ -63,7 +65,7 @@ struct FwdParams {
 struct __align__(8) Barriers {
   uint64_t q_full;
   uint64_t k_full[KS], k_empty[KS], v_full[VS], v_empty[VS];
-  uint64_t s_full[NQ], p_ready[NQ], o_full[NQ], o_empty[NQ];
+  uint64_t s_full[NQ], o_full[NQ];
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -94,8 +96,7 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
     for (int i = 0; i < KS; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1); }
     for (int i = 0; i < VS; ++i) { mbar_init(&bar.v_full[i], 1); mbar_init(&bar.v_empty[i], 1); }
     for (int i = 0; i < NQ; ++i) {
-      mbar_init(&bar.s_full[i], 1); mbar_init(&bar.p_ready[i], 128);
-      mbar_init(&bar.o_full[i], 1); mbar_init(&bar.o_empty[i], 128);
+      mbar_init(&bar.s_full[i], 1); mbar_init(&bar.o_full[i], 1);
     }
     fence_mbar_init();
   }
@@ -190,15 +191,16 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
           // one round of barrier tests per head: for head 0 also the V tile of this step and the K tile
           // of the next one (each separate wait would cost the issuing warp hundreds of cycles)
           if (q == 0) {
+            // the V tile of this step and the K tile of the next one first (they land while the warps
+            // still compute), then the hand-off of P through the named barrier
             const bool more = j + 1 < n_tiles;
             const int ksn = (j + 1) % KS;
-            ok = mbar_wait_all3(&bar.p_ready[0], j & 1, &bar.v_full[vs], (j / VS) & 1,
+            ok = mbar_wait_all3(&bar.v_full[vs], (j / VS) & 1, &bar.v_full[vs], (j / VS) & 1,
                                 more ? &bar.k_full[ksn] : &bar.v_full[vs], more ? ((j + 1) / KS) & 1 : (j / VS) & 1,
                                 abortp, p.status);
-          } else {
-            ok = mbar_wait_all1(&bar.p_ready[q], j & 1, abortp, p.status);
+            if (!ok) break;
           }
-          if (!ok) break;
+          named_sync(kBarP + q, kBarThreads);
           tc_fence_after();
           issue_pv(q, vs, j == 0);
           commit(&bar.o_full[q]);
@@ -231,6 +233,10 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       const bool diag = qt.causal && (j == n_tiles - 1);
       const int limit = diag ? min(row + 1, n_valid) : n_valid;  // keys [0, limit) are visible
       const bool need_mask = diag || n_valid < 128;
+      // A warp that gave up on a wait (ok == false) skips the tile's work but still arrives on the named
+      // barrier of every remaining tile, so that the MMA warp is never left waiting at one.
+      do {
+      if (!ok) break;
       // ---- softmax of this tile: the whole score row in one round trip to tensor memory ----
       ok = mbar_wait(&bar.s_full[q], j & 1, abortp, p.status);
       if (!ok) break;
@@ -341,8 +347,9 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
         fence_proxy_async();
       }
       tmem_wait_st();
+      } while (false);
       tc_fence_before();
-      mbar_arrive(&bar.p_ready[q]);
+      named_arrive(kBarP + q, kBarThreads);
     }
     // ---- last tile's product, normalise, store ----
     if (ok) ok = mbar_wait(&bar.o_full[q], (n_tiles - 1) & 1, abortp, p.status);

@@ -179,6 +179,21 @@ __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// ---------------------------------------------------------------- named barriers
+// Hand-off from the softmax warps to the MMA-issuing warp through a hardware named barrier: the
+// producers arrive (they do not wait), the consumer warp syncs.  A hop costs ~25 cycles against ~150
+// (idle SM) to ~300 (MMAs running) for an mbarrier in shared memory.  A named barrier has no phases
+// and no timeout, so it is only used where (a) the producers cannot arrive a second time before the
+// consumer has synced on the first (their next arrival depends on an MMA that the consumer issues
+// after that sync), and (b) every producer performs all its arrivals even after it gave up on a
+// wait of its own (see named_arrive_rest in the kernels), so the consumer is never left waiting.
+__device__ __forceinline__ void named_arrive(uint32_t id, uint32_t n_threads) {
+  asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+__device__ __forceinline__ void named_sync(uint32_t id, uint32_t n_threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+
 // ---------------------------------------------------------------- TMA
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
