@@ -41,8 +41,9 @@ constexpr int ST = 2;                              // (Q, dO) tile ring depth
 static_assert(kSubRows == 128, "the dK/dV kernel steps through 128-row query tiles");
 constexpr int kThreads = (8 + 2) * 32;             // 8 softmax-backward warps + producer + MMA
 constexpr uint32_t TM_ST = 0, TM_DPT = 128, TM_DV = 256, TM_DK = 384;
-// named barriers (softmax warps arrive, the MMA warp syncs): P^T(i) stored, dS^T(i) stored
-constexpr uint32_t kBarP = 1, kBarDs = 2, kBarThreads = 8 * 32 + 32;
+// named barriers (softmax warps arrive, the MMA warp syncs): dS^T(i) stored; quarters of P^T(i) stored
+// (dV starts on the first quarter while the warps still compute the rest)
+constexpr uint32_t kBarDs = 1, kBarP = 2, kBarThreads = 8 * 32 + 32;   // dS^T: id 1; P^T quarters: ids 2..5
 
 struct Maps {
   CUtensorMap q, d_o;  // boxes of 128 rows x 64 columns
@@ -281,14 +282,8 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
           mma_ss_lohi(d, ones_lo, kSliceDescHi, extra_lo, kSliceDescHi, idesc_kk, 1u);
         }
       };
-      auto mma_acc = [&](uint32_t d, uint32_t a_tmem, uint32_t b0, uint32_t acc0) {  // D += A[tmem] B, B MN-major
-        // packed bf16, 16 query rows per 8 columns; rows 0-63 at +0, rows 64-127 at +64
-        if (elect_one()) {
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            mma_ts_lo(d, a_tmem + (k >> 2) * 64 + (k & 3) * 8, b0 + k * 128, idesc_mn, k > 0 ? 1u : acc0);
-        }
-      };
+      // dV += P^T dO and dK += dS^T Q take A from tensor memory: packed bf16, 16 query rows per 8 columns,
+      // rows 0-63 at +0, rows 64-127 at +64; B (dO, Q) MN-major in shared memory, K = 16 slice k at + k * 128
       auto commit = [&](uint64_t* b) { if (elect_one()) mma_commit(b); };
       auto wait = [&](uint64_t* b, uint32_t parity) {
         return __all_sync(0xffffffffu, mbar_wait_relaxed(b, parity, abortp, p.status));
@@ -304,9 +299,16 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       for (int i = 0; ok && i < n_it; ++i) {
         const uint32_t so = (i % ST) * (kTileBytes >> 4), so1 = ((i + 1) % ST) * (kTileBytes >> 4);
         const uint32_t sx1 = ((i + 1) % ST) * (kSliceBytes >> 4);
-        named_sync(kBarP, kBarThreads);
-        tc_fence_after();
-        mma_acc(tmem + TM_DV, tmem + TM_ST, g_mn + so, i > 0);
+        // dV(i) in four quarters of two K = 16 slices each, as the quarters of P^T(i) arrive
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          named_sync(kBarP + g, kBarThreads);
+          tc_fence_after();
+          if (elect_one()) {
+            mma_ts_lo(tmem + TM_DV, tmem + TM_ST + g * 8, g_mn + so + g * 128, idesc_mn, g > 0 ? 1u : uint32_t(i > 0));
+            mma_ts_lo(tmem + TM_DV, tmem + TM_ST + 64 + g * 8, g_mn + so + (4 + g) * 128, idesc_mn, 1u);
+          }
+        }
         commit(&bar.do_empty[i % ST]);          // dO(i) is done with: its stage may take dO(i + ST)
         if (i + 1 < n_it) {
           // the Q tile of step i+1 arrives late (two-stage ring): wait behind dV(i), not before it
@@ -315,12 +317,19 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
           mma_kk(tmem + TM_ST, k_lo, q_lo + so1, lsex_lo + sx1);
           commit(&bar.s_full);
         }
-        // dS^T(i) stored; in the same round, dO(i+1) (it landed long ago: its stage was released early)
+        // dO(i+1) landed long ago (its stage was released early)
+        // dK(i) once all of dS^T(i) is stored (starting it on the first half measured slower: it is not on the
+        // step's critical path, and every extra sync delays the MMA warp a little)
         named_sync(kBarDs, kBarThreads);
         if (i + 1 < n_it) ok = wait(&bar.do_full[(i + 1) % ST], ((i + 1) / ST) & 1);
         if (!ok) break;
         tc_fence_after();
-        mma_acc(tmem + TM_DK, tmem + TM_DPT, q_mn + so, i > 0);
+        if (elect_one()) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            mma_ts_lo(tmem + TM_DK, tmem + TM_DPT + (k >> 2) * 64 + (k & 3) * 8, q_mn + so + k * 128, idesc_mn,
+                      k > 0 ? 1u : uint32_t(i > 0));
+        }
         commit(&bar.q_empty[i % ST]);
         if (i + 1 < n_it) {
           mma_kk(tmem + TM_DPT, v_lo, g_lo + so1, dlx_lo + sx1);
@@ -345,6 +354,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       // (a warp that gave up on a wait still walks the loop and performs every arrival on the named
       // barriers, so that the MMA warp is never left waiting at one)
       if (ok) ok = mbar_wait(&bar.s_full, i & 1, abortp, p.status);
+      int quarters_sent = 0;
       if (ok) {
         tc_fence_after();
         uint32_t s[2][32];
@@ -380,12 +390,15 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
             }
             pk[(g & 1) * 8 + (i >> 1)] = pack_bf16(p0, p1);
           }
-          if (g & 1) tmem_st16(t_lane + TM_ST + wg * 64 + (g >> 1) * 16, pk);
+          // 16 of the warp's 64 query rows are stored: dV may start on them
+          tmem_st8(t_lane + TM_ST + wg * 64 + g * 8, pk + (g & 1) * 8);
+          tmem_wait_st();
+          tc_fence_before();
+          named_arrive(kBarP + g, kBarThreads);
+          quarters_sent = g + 1;
         }
       }
-      tmem_wait_st();
-      tc_fence_before();
-      named_arrive(kBarP, kBarThreads);
+      for (int g = quarters_sent; g < 4; ++g) named_arrive(kBarP + g, kBarThreads);   // gave up on a wait
       // ---- half-step 2: dS^T = P^T o dP^T_aug (-D is already inside) ----
       if (ok) ok = mbar_wait(&bar.dp_full, i & 1, abortp, p.status);
       if (ok) {
