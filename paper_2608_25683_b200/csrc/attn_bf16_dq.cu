@@ -293,11 +293,13 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       // A warp stages only its own 32 rows: 272-byte pitch, no bank conflicts either way, no CTA barrier.
       constexpr int kPitch = 272;
       uint8_t* stage = sK + warp * (32 * kPitch);
+      uint32_t acc[4][32];   // the whole accumulator row in one round trip
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(t_lane + TM_DQ + c * 32, acc[c]);
+      tmem_wait_ld();
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(t_lane + TM_DQ + c * 32, r);
-        tmem_wait_ld();
+        uint32_t (&r)[32] = acc[c];
         if (qt.part_row0 < 0) {
 #pragma unroll
           for (int x = 0; x < 4; ++x) {
