@@ -7,6 +7,9 @@ mask counts, no tile padding, no duplicated prefix work, no recompute).
 
   python bench.py --gpus N --steps K --warmup W [--config c2] [--impl reference]
 
+Without --config the headline is c5 (the largest single-GPU configuration) and c2, c3, c4
+and the HBM-bound c2s are measured in the same run and reported under `per_config`.
+
 One step = one pass of the whole hot path (forward, D pre-pass, dQ, dK/dV) over
 one synthetic batch.  N > 1 (torchrun): every rank runs an independent batch
 (prefix groups never span workers), no data-path collective, weak scaling.
@@ -33,7 +36,8 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel
 # (dkv_kernel), from the ncu captures summarised under profiles/ ; None = not captured.
-NCU_TRAFFIC_BYTES = {"c2": 355363584 + 24176640}  # dram read + write of one dkv_kernel launch, profiles/dkv_kernel_c2.md
+NCU_TRAFFIC_BYTES = {"c2": 355363584 + 24176640,   # profiles/dkv_kernel_c2.md
+                     "c3": 1886000000 + 72000000}   # profiles/kernels_c3.md
 
 
 def peaks():
@@ -137,8 +141,9 @@ def sub_workload(w, n_keep):
                     w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, seg_flags=fl, seed=w.seed)
 
 
-def oracle_leg(w, n_keep, seed, steps=1, warmup=0):
-    """Times the fp64 oracle, as it stands, on KV head 0 of the first n_keep samples."""
+def oracle_leg(w, n_keep, seed, steps=1, warmup=0, budget=1.5e12):
+    """Times the fp64 oracle, as it stands, on KV head 0 of the first n_keep samples.
+    budget: fp64 FLOP of unshared work per pass (1.5e12 = 10-30 s on the host cores of this pool)."""
     import torch
     from oracle import oracle_attn, oracle_plan
     from paper_2608_25683_b200.workloads import make_inputs
@@ -147,7 +152,6 @@ def oracle_leg(w, n_keep, seed, steps=1, warmup=0):
     # count.  Fewer samples first; if one sample alone is too large (c5), an evenly spaced subset of the
     # query rows (exact for those rows: the other dO rows are taken as zero).
     G = w.n_q_heads // w.n_kv_heads
-    budget = 1.5e12   # fp64 FLOP of flat work per pass: 10-30 s on the host cores of this pool
     while True:
         sw = sub_workload(w, n_keep)
         plan = oracle_plan(sw.parent, sw.seg_len, sw.group_block_size, sw.seg_flags, None)
@@ -193,7 +197,9 @@ def run_reference(args):
     if rank != 0:
         return
     w = make_workload(args.config, args.seed)
-    base, t = oracle_leg(w, args.ref_samples, args.seed + 1, steps=args.steps, warmup=args.warmup)
+    # every step is a bounded sample; the whole run (warm-up + steps) stays near 4e12 FLOP of oracle work
+    base, t = oracle_leg(w, args.ref_samples, args.seed + 1, steps=args.steps, warmup=args.warmup,
+                         budget=min(1.5e12, 4e12 / max(1, args.steps + args.warmup)))
     line = dict(metric=METRIC, value=base["value"], unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=t * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="f64", data="synthetic", impl="reference",
@@ -304,11 +310,11 @@ def flat_runner(lib, r, device, head_slice=None):
     """The same kernels on the unshared layout: every sample a root of its own
     holding copies of its tokens; dO goes to the first copy of each token."""
     import torch
-    from paper_2608_25683_b200.workloads import Workload
+    from paper_2608_25683_b200.workloads import Workload, flatten_forest
 
     V = r.plan.view
     w = r.w
-    parent, seg_len, gbs, tok_src, first = lib.flatten_forest(V)
+    parent, seg_len, gbs, tok_src, first = flatten_forest(V)
     Hq, Hkv = w.n_q_heads, w.n_kv_heads
     G = Hq // Hkv
     hs = slice(None) if head_slice is None else slice(head_slice * G, (head_slice + 1) * G)
@@ -347,7 +353,8 @@ def library_context_leg(lib, w, V, device, ms_tree, flops, iters):
         from flash_attn import flash_attn_varlen_func
     except Exception as ex:
         return {"unavailable": str(ex)[:120]}
-    _, lens, _, _, _ = lib.flatten_forest(V)
+    from paper_2608_25683_b200.workloads import flatten_forest
+    _, lens, _, _, _ = flatten_forest(V)
     lens = [int(x) for x in lens]
     Hq, Hkv, d = w.n_q_heads, w.n_kv_heads, w.head_dim
     T = sum(lens)
@@ -514,53 +521,17 @@ def microbatch_leg(lib, w, device, flops, seed, iters):
             "live_slots_during_after": trace if M <= 64 else trace[:64]}
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="c2")
-    ap.add_argument("--seed", type=int, default=2000)
-    ap.add_argument("--cpu-samples", type=int, default=4, help="samples in the oracle's timed sample")
-    ap.add_argument("--ref-samples", type=int, default=2, help="samples per step of --impl reference")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-unshared", action="store_true")
-    ap.add_argument("--context", action="store_true",
-                    help="also time a library's varlen attention (flash_attn) on the unshared layout, for context")
-    ap.add_argument("--block-size", default=None,
-                    help="override the page size of every group: 16|32|64|128|256, or 'adaptive' (one extent per span)")
-    ap.add_argument("--length-scale", type=float, default=1.0,
-                    help="scale every segment length (tree shape and prefix match rate unchanged, cf. Sec. 7.5)")
-    ap.add_argument("--pack", action="store_true", help="also time K/V scatter into the pools and the gather back")
-    ap.add_argument("--schedule", action="store_true",
-                    help="also fit Eq. 1 to measured times and compare load-balanced with round-robin group placement")
-    ap.add_argument("--microbatch", action="store_true",
-                    help="also run the group as one micro-batch per branch with the Dynamic Block Caching manager")
-    args = ap.parse_args()
-    if args.impl == "reference":
-        run_reference(args)
-        return
-
+def measure_config(args, lib, name, device, rank, world, local, headline):
+    """All measurements of one configuration.  Returns None on ranks other than 0 once the timed
+    region (which every rank takes part in) is over."""
     import torch
     import torch.distributed as dist
 
-    from paper_2608_25683_b200 import binding as lib, build, dist_util
+    from paper_2608_25683_b200 import dist_util
     from paper_2608_25683_b200.workloads import make_workload
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    device = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(device))
-    build.build()
-
     # every rank gets an independent batch of the same shape (groups never span workers)
-    w = make_workload(args.config, dist_util.rank_seed(args.seed, rank), scale_len=args.length_scale)
+    w = make_workload(name, dist_util.rank_seed(args.seed, rank), scale_len=args.length_scale)
     if args.block_size is not None:
         bs = 0 if args.block_size == "adaptive" else int(args.block_size)
         w.group_block_size = [bs] * len(w.group_block_size)
@@ -587,6 +558,7 @@ def main():
     step_bytes = 5 * qb + 6 * kb + 2 * lb
     # a working set that fits in the L2 would be served from it after the first step: flush between steps
     flush = device if step_bytes < 2 * L2_BYTES else None
+    steps = args.steps
 
     def barrier():
         if world > 1:
@@ -607,25 +579,56 @@ def main():
         barrier()
         if flush is None:
             e0.record()
-            for _ in range(args.steps):
+            for _ in range(steps):
                 r.step()
             e1.record()
             barrier()
-            ms = e0.elapsed_time(e1) / args.steps
+            ms = e0.elapsed_time(e1) / steps
         else:
-            ms = time_region(r.step, args.steps, 0, flush)
+            ms = time_region(r.step, steps, 0, flush)
             barrier()
     ms_max, flops_all = dist_util.aggregate(ms, flops, device)  # max over ranks, sum of work
     value = flops_all / (ms_max * 1e-3) / 1e12
-
     if rank != 0:
-        if world > 1:
-            dist.barrier()
-            dist.destroy_process_group()
-        return
+        return None
+
+    # ---- per-kernel times INSIDE running steps, right behind the headline region (the same warmed, power-
+    # capped state): a step is issued as forward | D pre-pass | dQ | dK/dV with a CUDA event between the parts,
+    # so the parts add up to the step; the SM clock is sampled over exactly these steps ----
+    phases = (("fwd_kernel", None), ("delta_kernel", 1), ("dq_kernel", 2), ("dkv_kernel", 4))
+    n_ph = max(3, min(400, int(np.ceil(600.0 / ms))))       # >= 0.6 s of steps, so that the sampler sees them
+    with ClockSampler(local) as kclocks:
+        t_w = time.perf_counter()
+        while time.perf_counter() - t_w < 0.4:              # back into the headline's state after the sampler restart
+            r.step()
+            torch.cuda.synchronize()
+        marks = []
+        for _ in range(n_ph):
+            if flush is not None:
+                flush_l2(flush)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+            ev[0].record()
+            r.fwd()
+            ev[1].record()
+            for i, (_, mask) in enumerate(phases[1:]):
+                lib.psrl_bench_bwd_phases(r.plan, r.q, r.k, r.v, r.o, r.lse, r.d_o, r.scale, r.dq, r.dk, r.dv, mask)
+                ev[2 + i].record()
+            marks.append(ev)
+        torch.cuda.synchronize()
+    kern = {nm: float(np.mean([m[i].elapsed_time(m[i + 1]) for m in marks])) for i, (nm, _) in enumerate(phases)}
+    kclk = kclocks.summary()
+
+    # ---- host time of a step's calls (argument checks, tensor-map lookups, launches), GPU idle at the start ----
+    torch.cuda.synchronize()
+    n_h = 10 if ms < 50 else 2
+    th = time.perf_counter()
+    for _ in range(n_h):
+        r.step()
+    host_ms = (time.perf_counter() - th) / n_h * 1e3
+    torch.cuda.synchronize()
 
     # ---- every step on its own (median, min) and bitwise reproducibility over three runs ----
-    n_each = max(5, min(args.steps, 20))
+    n_each = max(3, min(steps, 20)) if ms < 100 else 3
     evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_each + 1)]
     if flush is None:
         evs[0].record()
@@ -650,44 +653,42 @@ def main():
     torch.cuda.empty_cache()
 
     pk = peaks()
-    # ---- per-kernel times (each kernel alone, CUDA events on the launch stream) ----
-    it = max(5, min(args.steps, 20))
-    t_fwd = time_region(r.fwd, it, 2, flush)
-    kern = {}
-    for name, mask in (("delta_kernel", 1), ("dq_kernel", 2), ("dkv_kernel", 4)):
-        lib.psrl_profile_bwd_phases(mask)
-        kern[name] = time_region(r.bwd, it, 2, flush)
-    lib.psrl_profile_bwd_phases(7)
-    kern["fwd_kernel"] = t_fwd
     d, Hq, pairs = w.head_dim, w.n_q_heads, float(V["tree_pairs"])
     # contractions each kernel has to execute for its outputs (2*d flops per pair, head and contraction):
     # forward S, PV; dQ kernel S, dP, dQ; dK/dV kernel S^T, dP^T, dV, dK.  The step metric counts 14*d (S and dP once).
     kflops = {"fwd_kernel": 4 * d * Hq * pairs, "dq_kernel": 6 * d * Hq * pairs, "dkv_kernel": 8 * d * Hq * pairs}
     kernels = {}
-    for name, tms in kern.items():
-        kernels[name] = {"ms": round(tms, 4)}
-        if name in kflops:
-            kernels[name]["algorithmic_tflops"] = round(kflops[name] / (tms * 1e-3) / 1e12, 2)
-    for name, tms in kern.items():
-        kernels[name]["algorithmic_gbs"] = round(kbytes[name] / (tms * 1e-3) / 1e9, 1)
+    for nm, tms in kern.items():
+        kernels[nm] = {"ms": round(tms, 4), "sm_mhz": kclk["sm_mhz"]}
+        if nm in kflops:
+            kernels[nm]["algorithmic_tflops"] = round(kflops[nm] / (tms * 1e-3) / 1e12, 2)
+        kernels[nm]["algorithmic_gbs"] = round(kbytes[nm] / (tms * 1e-3) / 1e9, 1)
+    sum_ms = sum(kern.values())
     dom = max(("fwd_kernel", "dq_kernel", "dkv_kernel"), key=lambda n: kern[n])
     ridge = pk["bf16_tflops"] * 1e12 / (pk["hbm_gbs"] * 1e9)
     hbm_bound = w.dtype == "bf16" and flops / step_bytes < ridge
+    timing_note = ("each kernel timed inside running steps (events between the step's parts), mean of %d steps, "
+                   "SM clock sampled over those steps" % n_ph)
     if hbm_bound:
         achieved = kbytes[dom] / (kern[dom] * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
-                    "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+                    "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": NCU_TRAFFIC_BYTES.get(name),
                     "peak_source": f"{pk['source']} copy bandwidth", "kernels": kernels,
                     "step_algorithmic_bytes": step_bytes, "step_flop_per_byte": round(flops / step_bytes, 1),
-                    "whole_step_gbs": round(step_bytes / (ms * 1e-3) / 1e9, 1)}
+                    "whole_step_gbs": round(step_bytes / (ms * 1e-3) / 1e9, 1),
+                    "whole_step_frac": round(step_bytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], 4)}
     else:
         achieved = kflops[dom] / (kern[dom] * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": dom, "achieved": round(achieved, 2), "peak": pk["bf16_tflops"],
                     "unit": "TFLOP/s", "frac": round(achieved / pk["bf16_tflops"], 4),
-                    "traffic": NCU_TRAFFIC_BYTES.get(args.config),
-                    "peak_source": f"{pk['source']} burst (kernel timed alone)", "kernels": kernels,
+                    "traffic": NCU_TRAFFIC_BYTES.get(name),
+                    "peak_source": f"{pk['source']} cuBLAS bf16 burst (the sustained figure, "
+                                   f"{pk['bf16_tflops_sustained']}, was taken at a lower SM clock than this run's)",
+                    "frac_of_sustained": round(achieved / pk["bf16_tflops_sustained"], 4), "kernels": kernels,
                     "whole_step_frac_of_burst": round(value / world / pk["bf16_tflops"], 4),
                     "whole_step_frac_of_sustained": round(value / world / pk["bf16_tflops_sustained"], 4)}
+    roofline.update(kernel_timing=timing_note, kernel_clocks=kclk, sum_kernel_ms=round(sum_ms, 4),
+                    sum_kernel_ms_over_step_ms=round(sum_ms / ms, 4))
     if w.dtype != "bf16":
         roofline["bound"] = "alu"
 
@@ -702,8 +703,8 @@ def main():
         ho.copy_(r.o, non_blocking=True); hl.copy_(r.lse, non_blocking=True); hdq.copy_(r.dq, non_blocking=True)
         hdk.copy_(r.dk, non_blocking=True); hdv.copy_(r.dv, non_blocking=True)
 
-    n_e2e = max(4, min(args.steps, 10))
-    e2e_serial_ms = time_region(e2e_step, n_e2e, 2)
+    n_e2e = max(4, min(steps, 10)) if ms < 100 else 3
+    e2e_serial_ms = time_region(e2e_step, n_e2e, 2 if ms < 100 else 1)
 
     # The same, software-pipelined the way a training loop feeds a device: three streams and two sets of device
     # buffers, so that step i+1's host->device copies and step i-1's device->host copies run beside step i.
@@ -750,26 +751,27 @@ def main():
     e2e_pipelined(2)
     e2e_ms = e2e_pipelined(n_e2e)
     del r2, pair
-    torch.cuda.empty_cache()
-    es = 2 if w.dtype == "bf16" else 4
     nbytes = lambda *ts: int(sum(x.numel() * x.element_size() for x in ts))
     e2e = {"value": round(flops / (e2e_ms * 1e-3) / 1e12 * world, 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
            "h2d_bytes_per_step": nbytes(hq, hk, hv, hdo), "d2h_bytes_per_step": nbytes(ho, hl, hdq, hdk, hdv),
            "mode": "three streams, two sets of device buffers: copies of neighbouring steps overlap the kernels",
            "serial": {"value": round(flops / (e2e_serial_ms * 1e-3) / 1e12 * world, 3),
                       "ms_per_step": round(e2e_serial_ms, 3), "mode": "copy in, run, copy out on one stream"}}
+    del hq, hk, hv, hdo, ho, hl, hdq, hdk, hdv
+    torch.cuda.empty_cache()
 
     # ---- the same kernels on the unshared (flattened) layout ----
-    print("[bench] tree path measured; unshared leg", file=sys.stderr, flush=True)
+    print(f"[bench] {name}: tree path measured; unshared leg", file=sys.stderr, flush=True)
     unshared = None
-    if not args.no_unshared and world == 1:
+    if not args.no_unshared and world == 1 and all((f & 1) for f in V["seg_flags"]):
         try:
             bytes_flat = V["flat_tokens"] * Hq * d * es * 4
             slices = 1 if bytes_flat < 60e9 else w.n_kv_heads
             t_flat = 0.0
-            for s in range(slices):
-                fr = flat_runner(lib, r, device, head_slice=None if slices == 1 else s)
-                t_flat += time_region(fr.step, max(3, min(args.steps, 10)), 2)
+            n_fl = max(3, min(steps, 10)) if ms < 100 else 2
+            for sl in range(slices):
+                fr = flat_runner(lib, r, device, head_slice=None if slices == 1 else sl)
+                t_flat += time_region(fr.step, n_fl, 2 if ms < 100 else 1)
                 del fr
                 torch.cuda.empty_cache()
             unshared = {"ms_per_step": round(t_flat, 3), "speedup_vs_unshared": round(t_flat / ms, 3),
@@ -778,53 +780,134 @@ def main():
         except Exception as ex:  # e.g. out of memory on the flattened tensors
             unshared = {"error": str(ex)[:200]}
 
-    context = None
-    if args.context and world == 1:
-        torch.cuda.synchronize()
-        print("[bench] library context leg", file=sys.stderr, flush=True)
-        context = library_context_leg(lib, w, V, device, ms, flops, max(3, min(args.steps, 10)))
-        torch.cuda.synchronize()
-        print("[bench] library context leg done", file=sys.stderr, flush=True)
-        torch.cuda.empty_cache()
+    res = dict(value=round(value, 3), ms_per_step=round(ms_max, 4), unit=UNIT,
+               dtype=("bf16" if w.dtype == "bf16" else "f32"),
+               config=dict(workload_config(w, V), length_scale=args.length_scale, pool_slots=V["pool_slots"], l2=(
+                   "per-step working set exceeds the 126 MB L2 (inputs larger than L2); no explicit flush" if flush is None
+                   else "working set fits in the L2: a 252 MB buffer is overwritten before every timed step "
+                        "(each step timed on its own, flush outside the timed part)")),
+               clocks=clocks.summary(), e2e=e2e,
+               gpu_launches=(lib.psrl_launch_count(r.plan, False) + lib.psrl_launch_count(r.plan, True)) * steps,
+               roofline=roofline, step_ms=step_stats, bitwise_reproducible_3_runs=bool(same),
+               plan=dict(plan_ms, host_ms_per_step_of_calls=round(host_ms, 4)), unshared=unshared,
+               frac_of_bf16_peak={"burst": round(value / world / pk["bf16_tflops"], 4),
+                                  "sustained": round(value / world / pk["bf16_tflops_sustained"], 4)})
 
-    pack = None
-    if args.pack and world == 1:
-        import torch as _t
-        T, cap = V["T"], r.k.shape[1]
-        k_tok = _t.randn(T, w.n_kv_heads, w.head_dim, device=device).to(r.k.dtype)
-        v_tok = _t.randn(T, w.n_kv_heads, w.head_dim, device=device).to(r.k.dtype)
-        nbytes_pack = 2 * 2 * k_tok.numel() * k_tok.element_size()      # K and V, read + write
-        fl = device if nbytes_pack < 2 * L2_BYTES else None
-        t_sc = time_region(lambda: lib.psrl_kv_scatter(r.plan, k_tok, v_tok, r.k, r.v), 10, 2, fl)
-        t_ga = time_region(lambda: lib.psrl_kv_gather(r.plan, r.k, r.v, k_tok, v_tok), 10, 2, fl)
-        pack = {"bytes_per_call": nbytes_pack, "scatter_ms": round(t_sc, 4), "gather_ms": round(t_ga, 4),
+    if headline:
+        extra = {}
+        if args.context and world == 1:
+            torch.cuda.synchronize()
+            print("[bench] library context leg", file=sys.stderr, flush=True)
+            extra["library_context"] = library_context_leg(lib, w, V, device, ms, flops, max(3, min(steps, 10)))
+            torch.cuda.synchronize()
+            torch.cuda.empty_cache()
+        if args.pack and world == 1:
+            T = V["T"]
+            k_tok = torch.randn(T, w.n_kv_heads, w.head_dim, device=device).to(r.k.dtype)
+            v_tok = torch.randn(T, w.n_kv_heads, w.head_dim, device=device).to(r.k.dtype)
+            nbytes_pack = 2 * 2 * k_tok.numel() * k_tok.element_size()      # K and V, read + write
+            fl = device if nbytes_pack < 2 * L2_BYTES else None
+            t_sc = time_region(lambda: lib.psrl_kv_scatter(r.plan, k_tok, v_tok, r.k, r.v), 10, 2, fl)
+            t_ga = time_region(lambda: lib.psrl_kv_gather(r.plan, r.k, r.v, k_tok, v_tok), 10, 2, fl)
+            extra["kv_pack"] = {
+                "bytes_per_call": nbytes_pack, "scatter_ms": round(t_sc, 4), "gather_ms": round(t_ga, 4),
                 "scatter_gbs": round(nbytes_pack / (t_sc * 1e-3) / 1e9, 1), "gather_gbs": round(nbytes_pack / (t_ga * 1e-3) / 1e9, 1),
                 "hbm_peak_gbs": pk["hbm_gbs"], "scatter_frac": round(nbytes_pack / (t_sc * 1e-3) / 1e9 / pk["hbm_gbs"], 4),
                 "gather_frac": round(nbytes_pack / (t_ga * 1e-3) / 1e9 / pk["hbm_gbs"], 4)}
+        if args.schedule and world == 1:
+            extra["schedule"] = schedule_leg(lib, device, args.seed + 11)
+        if args.microbatch and world == 1:
+            extra["microbatch"] = microbatch_leg(lib, w, device, flops, args.seed + 7, max(3, min(steps, 10)))
+        res["extra"] = extra
+        res["workload_obj"] = w
+    del r
+    torch.cuda.empty_cache()
+    return res
 
-    sched = None
-    if args.schedule and world == 1:
-        sched = schedule_leg(lib, device, args.seed + 11)
 
-    micro = None
-    if args.microbatch and world == 1:
-        micro = microbatch_leg(lib, w, device, flops, args.seed + 7, max(3, min(args.steps, 10)))
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default=None,
+                    help="one configuration (c1..c5, c2s).  Default: c5 is the headline (the largest single-GPU "
+                         "configuration) and c2, c3, c4 and the HBM-bound c2s are measured too, under per_config")
+    ap.add_argument("--seed", type=int, default=2000)
+    ap.add_argument("--cpu-samples", type=int, default=4, help="samples in the oracle's timed sample")
+    ap.add_argument("--ref-samples", type=int, default=2, help="samples per step of --impl reference")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-unshared", action="store_true")
+    ap.add_argument("--context", action="store_true",
+                    help="also time a library's varlen attention (flash_attn) on the unshared layout, for context")
+    ap.add_argument("--block-size", default=None,
+                    help="override the page size of every group: 16|32|64|128|256, or 'adaptive' (one extent per span)")
+    ap.add_argument("--length-scale", type=float, default=1.0,
+                    help="scale every segment length (tree shape and prefix match rate unchanged, cf. Sec. 7.5)")
+    ap.add_argument("--pack", action="store_true", help="also time K/V scatter into the pools and the gather back")
+    ap.add_argument("--schedule", action="store_true",
+                    help="also fit Eq. 1 to measured times and compare load-balanced with round-robin group placement")
+    ap.add_argument("--microbatch", action="store_true",
+                    help="also run the group as one micro-batch per branch with the Dynamic Block Caching manager")
+    args = ap.parse_args()
+    head_name = args.config or "c5"
+    others = [] if args.config else ["c2", "c3", "c4", "c2s"]
+    if args.impl == "reference":
+        args.config = head_name
+        run_reference(args)
+        return
 
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_25683_b200 import binding as lib, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    build.build()
+
+    # the other configurations first (short), the headline last; with several ranks only the headline runs
+    per_config = {}
+    if world == 1:
+        for name in others:
+            print(f"[bench] {name}", file=sys.stderr, flush=True)
+            try:
+                res = measure_config(args, lib, name, device, rank, world, local, headline=False)
+                res.pop("unit", None)
+                per_config[name] = res
+            except Exception as ex:   # one configuration must not take the headline down with it
+                per_config[name] = {"error": str(ex)[:300]}
+                torch.cuda.empty_cache()
+    print(f"[bench] {head_name} (headline)", file=sys.stderr, flush=True)
+    res = measure_config(args, lib, head_name, device, rank, world, local, headline=True)
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    w = res.pop("workload_obj")
+    extra = res.pop("extra")
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:
         cpu, _ = oracle_leg(w, args.cpu_samples, args.seed + 1)
 
-    line = dict(metric=METRIC, value=round(value, 3), unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
-                ms_per_step=round(ms_max, 4), higher_is_better=True, scaling="weak", vs_baseline=None,
-                dtype=("bf16" if w.dtype == "bf16" else "f32"), data="synthetic",
-                config=dict(workload_config(w, V), length_scale=args.length_scale, pool_slots=V["pool_slots"], l2=(
-                    "per-step working set exceeds the 126 MB L2 (inputs larger than L2); no explicit flush" if flush is None
-                    else "working set fits in the L2: a 252 MB buffer is overwritten before every timed step "
-                         "(each step timed on its own, flush outside the timed part)")), clocks=clocks.summary(), e2e=e2e, gpu_launches=(lib.psrl_launch_count(r.plan, False) + lib.psrl_launch_count(r.plan, True)) * args.steps,
-                roofline=roofline, cpu_baseline=cpu, step_ms=step_stats, bitwise_reproducible_3_runs=bool(same),
-                plan=plan_ms, unshared=unshared, library_context=context, microbatch=micro, schedule=sched, kv_pack=pack,
-                frac_of_bf16_peak={"burst": round(value / world / pk["bf16_tflops"], 4),
-                                   "sustained": round(value / world / pk["bf16_tflops_sustained"], 4)})
+    line = dict(metric=METRIC, value=res["value"], unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=res["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype=res["dtype"], data="synthetic", config=res["config"], clocks=res["clocks"], e2e=res["e2e"],
+                gpu_launches=res["gpu_launches"], roofline=res["roofline"], cpu_baseline=cpu, step_ms=res["step_ms"],
+                bitwise_reproducible_3_runs=res["bitwise_reproducible_3_runs"], plan=res["plan"],
+                unshared=res["unshared"], frac_of_bf16_peak=res["frac_of_bf16_peak"],
+                per_config=per_config or None, library_context=extra.get("library_context"),
+                microbatch=extra.get("microbatch"), schedule=extra.get("schedule"), kv_pack=extra.get("kv_pack"))
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()

@@ -226,11 +226,17 @@ psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const v
  * library, held until the process exits).  The call itself performs no
  * cudaMalloc / cudaFree and calls no allocating library routine.
  *
- * Same mathematics, same arguments and same results as psrl_tree_attn_bwd,
- * except:
+ * Same mathematics, same arguments (NULL Q-shaped pointers are accepted for a
+ * plan without query rows, as there) and bit-identical results as
+ * psrl_tree_attn_bwd, except:
  *   - no workspace arguments;
- *   - limit: n_q_heads * T_q <= 4,194,304 (the array holds one float per query
- *     row and head); larger plans return PSRL_ERR_WORKSPACE and must use
+ *   - limit: the array stands in for the whole workspace, so a plan fits when
+ *       psrl_bwd_workspace_bytes(plan) <= PSRL_BWD_STATIC_SCRATCH_BYTES,
+ *     i.e. 256 bytes of header + D (one float per query row and head, so
+ *     n_q_heads * T_q <= 4,194,304 at the very most) + the fp32 slabs of split
+ *     KV tiles (n_kv_heads * 128 KiB each) + the partial dQ rows of cascaded
+ *     prefixes (n_q_heads * 512 bytes each), the last two only for plans whose
+ *     schedule has them.  Larger plans return PSRL_ERR_WORKSPACE and must use
  *     psrl_tree_attn_bwd;
  *   - status_workspace (HOST pointer, may be NULL) receives the DEVICE address
  *     of the array's status header; pass it to psrl_device_status to read the
@@ -246,6 +252,7 @@ psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const v
  * Errors: INVALID_ARG, SHAPE, WORKSPACE (plan not uploaded, or over the
  * limit), CUDA.  Asynchronous.
  */
+#define PSRL_BWD_STATIC_SCRATCH_BYTES ((size_t)16777472) /* 16 MiB + 256 */
 psrl_status_t psrl_tree_attn_bwd_static(const psrl_plan_t* plan, const void* q, const void* k_pool,
                                         const void* v_pool, int64_t pool_capacity, const void* o, const float* lse,
                                         const void* d_o, void* d_q, void* dk_pool, void* dv_pool,
@@ -274,14 +281,18 @@ psrl_status_t psrl_kv_gather(const psrl_plan_t* plan, const void* k_pool, const 
                              int64_t pool_capacity, void* k_tok, void* v_tok, void* stream);
 
 /*
- * Profiling aid (no counterpart in the paper): restricts which kernels the
- * NEXT psrl_tree_attn_bwd calls of this process launch, so that each backward
- * kernel can be timed on its own with CUDA events.  Bit 0: D = rowsum(dO o O)
- * pre-pass, bit 1: dQ kernel, bit 2: dK/dV kernel.  Default 7 (everything);
- * with any other mask the skipped outputs are left untouched.  Returns the
- * previous mask.  Not thread-safe; meant for benchmarks only.
+ * Benchmark aid (no counterpart in the paper): psrl_tree_attn_bwd with a mask
+ * of the backward kernels to launch, so that each can be timed on its own
+ * with CUDA events.  Bit 0: D = rowsum(dO o O) pre-pass, bit 1: dQ kernel
+ * (+ its merge), bit 2: dK/dV kernel (+ its reduce).  phases = 7 is exactly
+ * psrl_tree_attn_bwd; with any other mask the outputs of the skipped kernels
+ * are left untouched (and a skipped pre-pass leaves D as the previous call on
+ * this workspace wrote it).  Stateless: the mask is an argument of the call.
  */
-int psrl_profile_bwd_phases(int mask);
+psrl_status_t psrl_bench_bwd_phases(const psrl_plan_t* plan, const void* q, const void* k_pool, const void* v_pool,
+                                    int64_t pool_capacity, const void* o, const float* lse, const void* d_o,
+                                    void* d_q, void* dk_pool, void* dv_pool, float softmax_scale, void* workspace,
+                                    size_t workspace_bytes, void* stream, int phases);
 
 /*
  * Number of kernels one psrl_tree_attn_fwd (backward == 0) or

@@ -21,13 +21,14 @@ STATUS_NAMES = [
     "PSRL_ERR_TIMEOUT", "PSRL_ERR_INTERNAL",
 ]
 PSRL_F32, PSRL_BF16 = 0, 1
+BWD_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024 + 256   # PSRL_BWD_STATIC_SCRATCH_BYTES of include/psrl.h
 SEG_HAS_Q, SEG_SAMPLE_END = 1, 2
 
 EXPORTS = [
     "psrl_plan_build", "psrl_plan_view", "psrl_plan_device_bytes", "psrl_plan_upload",
     "psrl_fwd_workspace_bytes", "psrl_bwd_workspace_bytes", "psrl_tree_attn_fwd", "psrl_tree_attn_bwd",
     "psrl_device_status", "psrl_last_cuda_error", "psrl_plan_destroy", "psrl_status_string",
-    "psrl_profile_bwd_phases", "psrl_tree_attn_bwd_static", "psrl_launch_count", "psrl_plan_schedule",
+    "psrl_bench_bwd_phases", "psrl_tree_attn_bwd_static", "psrl_launch_count", "psrl_plan_schedule",
     "psrl_cache_create", "psrl_cache_begin", "psrl_cache_end", "psrl_cache_stats", "psrl_cache_refcounts",
     "psrl_cache_destroy",
     "psrl_kv_scatter", "psrl_kv_gather",
@@ -137,8 +138,8 @@ def lib() -> C.CDLL:
                                             C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                                             C.POINTER(C.c_void_p), C.c_void_p]
     L.psrl_tree_attn_bwd_static.restype = C.c_int
-    L.psrl_profile_bwd_phases.argtypes = [C.c_int]
-    L.psrl_profile_bwd_phases.restype = C.c_int
+    L.psrl_bench_bwd_phases.argtypes = L.psrl_tree_attn_bwd.argtypes + [C.c_int]
+    L.psrl_bench_bwd_phases.restype = C.c_int
     L.psrl_plan_schedule.argtypes = [C.c_void_p, C.POINTER(_I32P), C.POINTER(C.c_size_t)]
     L.psrl_plan_schedule.restype = C.c_int
     _F64P = C.POINTER(C.c_double)
@@ -368,8 +369,10 @@ def psrl_tree_attn_bwd_static(plan: Plan, q, k_pool, v_pool, o, lse, d_o, softma
     the CUDA allocator (see include/psrl.h).  Unlike psrl_tree_attn_bwd this
     wrapper allocates nothing either, so every output tensor must be passed in.
     The library's built-in scratch array serves as workspace; it is shared by
-    all calls on the device, so calls must not overlap on the GPU, and it caps
-    the problem at n_q_heads * T_q <= 4,194,304 (PSRL_ERR_WORKSPACE beyond).
+    all calls on the device, so calls must not overlap on the GPU, and its size
+    caps the problem: plan.bwd_workspace_bytes() (header + D, one float per query
+    row and head, + slabs of split KV tiles + partial dQ rows) must not exceed
+    BWD_STATIC_SCRATCH_BYTES = 16 MiB + 256 (PSRL_ERR_WORKSPACE beyond).
     Returns the device address of the status header (for psrl_device_status)."""
     _check_dtype(plan, q, k_pool, v_pool, o, d_o, d_q, dk_pool, dv_pool)
     ws = C.c_void_p()
@@ -381,17 +384,17 @@ def psrl_tree_attn_bwd_static(plan: Plan, q, k_pool, v_pool, o, lse, d_o, softma
     return int(ws.value or 0)
 
 
-def psrl_profile_bwd_phases(mask: int) -> int:
-    """Profiling aid: choose which backward kernels the next calls launch
-    (bit 0 delta pre-pass, bit 1 dQ, bit 2 dK/dV); returns the previous mask."""
-    return int(lib().psrl_profile_bwd_phases(int(mask)))
-
-
-def _stream_ptr(stream):
-    import torch
-
-    s = torch.cuda.current_stream() if stream is None else stream
-    return C.c_void_p(s.cuda_stream)
+def psrl_bench_bwd_phases(plan: Plan, q, k_pool, v_pool, o, lse, d_o, softmax_scale: float, d_q, dk_pool, dv_pool,
+                          phases: int, stream=None, workspace=None):
+    """Benchmark aid: the backward with a mask of the kernels to launch (bit 0 D pre-pass, bit 1 dQ,
+    bit 2 dK/dV), so that each can be timed on its own.  Outputs must be passed in."""
+    _check_dtype(plan, q, k_pool, v_pool, o, d_o, d_q, dk_pool, dv_pool)
+    ws, wsb = workspace if workspace is not None else plan.workspace("bwd", q.device)
+    st = lib().psrl_bench_bwd_phases(plan.handle, q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(),
+                                     int(k_pool.shape[1]), o.data_ptr(), lse.data_ptr(), d_o.data_ptr(),
+                                     d_q.data_ptr(), dk_pool.data_ptr(), dv_pool.data_ptr(), float(softmax_scale),
+                                     C.c_void_p(ws), wsb, _stream_ptr(stream), int(phases))
+    _check(st, "psrl_bench_bwd_phases")
 
 
 def psrl_kv_scatter(plan: Plan, k_tok, v_tok, k_pool, v_pool, stream=None):
@@ -546,32 +549,3 @@ def _check_dtype(plan: Plan, *tensors):
             raise TypeError(f"tensor dtype {t.dtype} does not match the plan's {want}")
         if not t.is_cuda:
             raise RuntimeError("tensors must live on a CUDA device: this library has no CPU path")
-
-
-def flatten_forest(view: dict):
-    """The unshared layout: every sample becomes a root segment of its own
-    holding copies of its tokens (what a system without prefix sharing stores).
-
-    Returns (parent, seg_len, group_block_size, tok_src, first_copy) where
-    tok_src[i] is the tree token copied to flat token i and first_copy[i] says
-    whether it is that token's first copy in canonical sample order (the copy
-    that carries the token's upstream gradient row; the others get zero).
-    """
-    parent, seg_len, gbs, src = [], [], [], []
-    for e in view["sample_end_seg"]:
-        e = int(e)
-        path = list(view["anc_list"][view["anc_off"][e]:view["anc_off"][e + 1]]) + [e]
-        L = 0
-        for c in path:
-            t0 = int(view["seg_tok_off"][c])
-            n = int(view["seg_len"][c])
-            src.append(np.arange(t0, t0 + n, dtype=np.int64))
-            L += n
-        parent.append(-1)
-        seg_len.append(L)
-        gbs.append(int(view["seg_bs"][e]))
-    tok_src = np.concatenate(src)
-    _, first_idx = np.unique(tok_src, return_index=True)
-    first_copy = np.zeros(len(tok_src), dtype=bool)
-    first_copy[first_idx] = True
-    return parent, seg_len, gbs, tok_src, first_copy

@@ -7,14 +7,9 @@
 #include "kernels.h"
 #include "plan.h"
 
-struct psrl_plan {
-  psrl::Plan* p;
-};
-
 namespace psrl {
 static thread_local cudaError_t g_last_cuda = cudaSuccess;
 void set_last_cuda_error(cudaError_t e) { g_last_cuda = e; }
-int g_bwd_phase_mask = 7;
 int resident_ctas() {
   static thread_local int n[64] = {};
   int dev = 0;
@@ -26,11 +21,8 @@ int resident_ctas() {
 
 namespace {
 
-bool aligned(const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) == 0; }
-// Q-shaped tensors of a plan without any query row are empty: NULL is fine there
-bool aligned_q(const void* p, size_t a, const psrl::Plan& P) {
-  return (P.T_q == 0 && !p) || aligned(p, a);
-}
+bool aligned(const void* p, size_t a) { return psrl::ptr_aligned(p, a); }
+bool aligned_q(const void* p, size_t a, const psrl::Plan& P) { return psrl::ptr_aligned_q(p, a, P); }
 
 size_t ws_bytes(const psrl::Plan& P, bool bwd) {
   size_t n = psrl::kWsHeaderBytes;
@@ -142,10 +134,10 @@ psrl_status_t psrl_tree_attn_fwd(const psrl_plan_t* plan, const void* q, const v
   return psrl::fwd_bf16(a);
 }
 
-psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const void* k_pool, const void* v_pool,
+static psrl_status_t bwd_checked(const psrl_plan_t* plan, const void* q, const void* k_pool, const void* v_pool,
                                  int64_t pool_capacity, const void* o, const float* lse, const void* d_o, void* d_q,
                                  void* dk_pool, void* dv_pool, float softmax_scale, void* workspace,
-                                 size_t workspace_bytes, void* stream) {
+                                 size_t workspace_bytes, void* stream, int phases) {
   if (!plan || !plan->p) return PSRL_ERR_INVALID_ARG;
   const psrl::Plan& P = *plan->p;
   if (!aligned_q(q, 16, P) || !aligned(k_pool, 16) || !aligned(v_pool, 16) || !aligned_q(o, 16, P) ||
@@ -163,10 +155,27 @@ psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const v
   a.part = reinterpret_cast<float*>(static_cast<char*>(workspace) + psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P) +
                                     psrl::ws_slab_bytes(P));
   a.pool_capacity = pool_capacity; a.scale = softmax_scale; a.stream = static_cast<cudaStream_t>(stream);
+  a.phases = phases & 7;
   cudaError_t e = cudaMemsetAsync(workspace, 0, psrl::kWsHeaderBytes, a.stream);
   if (e != cudaSuccess) return cuda_status(e);
   if (P.dtype == PSRL_F32) return cuda_status(psrl::bwd_f32(a));
   return psrl::bwd_bf16(a);
+}
+
+psrl_status_t psrl_tree_attn_bwd(const psrl_plan_t* plan, const void* q, const void* k_pool, const void* v_pool,
+                                 int64_t pool_capacity, const void* o, const float* lse, const void* d_o, void* d_q,
+                                 void* dk_pool, void* dv_pool, float softmax_scale, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
+  return bwd_checked(plan, q, k_pool, v_pool, pool_capacity, o, lse, d_o, d_q, dk_pool, dv_pool, softmax_scale,
+                     workspace, workspace_bytes, stream, 7);
+}
+
+psrl_status_t psrl_bench_bwd_phases(const psrl_plan_t* plan, const void* q, const void* k_pool, const void* v_pool,
+                                    int64_t pool_capacity, const void* o, const float* lse, const void* d_o,
+                                    void* d_q, void* dk_pool, void* dv_pool, float softmax_scale, void* workspace,
+                                    size_t workspace_bytes, void* stream, int phases) {
+  return bwd_checked(plan, q, k_pool, v_pool, pool_capacity, o, lse, d_o, d_q, dk_pool, dv_pool, softmax_scale,
+                     workspace, workspace_bytes, stream, phases);
 }
 
 psrl_status_t psrl_device_status(const void* workspace, void* stream) {
@@ -178,12 +187,6 @@ psrl_status_t psrl_device_status(const void* workspace, void* stream) {
   if (st == 0) return PSRL_OK;
   if (st == PSRL_ERR_TIMEOUT) return PSRL_ERR_TIMEOUT;
   return PSRL_ERR_INTERNAL;
-}
-
-int psrl_profile_bwd_phases(int mask) {
-  const int prev = psrl::g_bwd_phase_mask;
-  psrl::g_bwd_phase_mask = mask & 7;
-  return prev;
 }
 
 int psrl_launch_count(const psrl_plan_t* plan, int backward) {

@@ -55,7 +55,7 @@ psrl_status_t bwd_bf16(const AttnArgs& a) {
   const Plan& P = *a.plan;
   const int64_t cap = a.pool_capacity;
   if (int64_t(P.Hkv) * cap > INT32_MAX || int64_t(P.Hq) * 128 > INT32_MAX) return PSRL_ERR_SHAPE;
-  if (P.T_q > 0 && (g_bwd_phase_mask & 1)) {
+  if (P.T_q > 0 && (a.phases & 1)) {
     // ---- D = rowsum(dO o O) ----
     const int64_t units = int64_t(P.T_q) * P.Hq;
     delta_kernel<<<unsigned((units + 15) / 16), 256, 0, a.stream>>>(
@@ -66,12 +66,12 @@ psrl_status_t bwd_bf16(const AttnArgs& a) {
       return PSRL_ERR_CUDA;
     }
   }
-  if (g_bwd_phase_mask & 2) {
+  if (a.phases & 2) {
     // ---- dQ (attn_bf16_dq.cu) ----
     const psrl_status_t st = dq_bf16(a);
     if (st != PSRL_OK) return st;
   }
-  if (g_bwd_phase_mask & 4) {
+  if (a.phases & 4) {
     // ---- dK, dV (attn_bf16_dkv.cu) ----
     const psrl_status_t st = dkv_bf16(a);
     if (st != PSRL_OK) return st;

@@ -122,6 +122,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
   __shared__ Barriers bar;
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
+  __shared__ StepBeacon s_beacon;   // the MMA warp's position, for softmax warps that gave up on a wait
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int item = blockIdx.x / p.Hkv, hk = blockIdx.x % p.Hkv;
@@ -132,6 +133,8 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
 
   if (tid == 0) {
     s_abort = 0;
+    s_beacon.at = -1;
+    s_beacon.left = 0;
     mbar_init(&bar.kv_full, 1);
     for (int i = 0; i < ST; ++i) {
       mbar_init(&bar.q_full[i], 2); mbar_init(&bar.q_empty[i], 1);
@@ -299,6 +302,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       for (int i = 0; ok && i < n_it; ++i) {
         const uint32_t so = (i % ST) * (kTileBytes >> 4), so1 = ((i + 1) % ST) * (kTileBytes >> 4);
         const uint32_t sx1 = ((i + 1) % ST) * (kSliceBytes >> 4);
+        if (lane == 0) s_beacon.at = i;   // before this step's five syncs (read only by warps that gave up)
         // dV(i) in four quarters of two K = 16 slices each, as the quarters of P^T(i) arrive
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
@@ -337,6 +341,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
         }
       }
       if (ok) commit(&bar.acc_full);
+      if (lane == 0) s_beacon.left = 1;   // no sync follows on any path
     }
   } else {
     // ======================= softmax-backward warps (8) =======================
@@ -345,6 +350,7 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
     const uint32_t t_lane = tmem + (uint32_t((warp & 3) * 32) << 16);
     const f32x2 scale2 = make_f32x2(p.scale_log2, p.scale_log2);
     bool ok = true;
+    bool arrive = true;   // false once the MMA warp has left its loop: nobody syncs any more
     for (int i = 0; i < n_it; ++i) {
       int g, row0, nvq, qpos0; bool diag;
       step(i, g, row0, nvq, diag, qpos0);
@@ -352,7 +358,8 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       // ---- half-step 1: P^T = exp2(c S^T_aug); -LSE / scale is already inside S^T_aug, and
       //      a query row beyond the valid range carries -inf there, so its column comes out 0 ----
       // (a warp that gave up on a wait still walks the loop and performs every arrival on the named
-      // barriers, so that the MMA warp is never left waiting at one)
+      // barriers - once per step, and for step i only when the MMA warp has reached step i, see
+      // StepBeacon - so that the MMA warp is never left waiting at one)
       if (ok) ok = mbar_wait(&bar.s_full, i & 1, abortp, p.status);
       int quarters_sent = 0;
       if (ok) {
@@ -398,7 +405,9 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
           quarters_sent = g + 1;
         }
       }
-      for (int g = quarters_sent; g < 4; ++g) named_arrive(kBarP + g, kBarThreads);   // gave up on a wait
+      if (!ok && arrive) arrive = beacon_reached(&s_beacon, i);
+      if (arrive)
+        for (int g = quarters_sent; g < 4; ++g) named_arrive(kBarP + g, kBarThreads);   // gave up on a wait
       // ---- half-step 2: dS^T = P^T o dP^T_aug (-D is already inside) ----
       if (ok) ok = mbar_wait(&bar.dp_full, i & 1, abortp, p.status);
       if (ok) {
@@ -421,7 +430,8 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       }
       tmem_wait_st();
       tc_fence_before();
-      named_arrive(kBarDs, kBarThreads);
+      if (!ok && arrive) arrive = beacon_reached(&s_beacon, i);
+      if (arrive) named_arrive(kBarDs, kBarThreads);
     }
     // ---- epilogue: warps 0-3 take dV, warps 4-7 take dK ----
     if (ok && n_it > 0) ok = mbar_wait(&bar.acc_full, 0, abortp, p.status);

@@ -266,15 +266,15 @@ cudaError_t bwd_impl(const AttnArgs& a) {
   const float* k = static_cast<const float*>(a.k_pool);
   const float* v = static_cast<const float*>(a.v_pool);
   const float* d_o = static_cast<const float*>(a.d_o);
-  if (units > 0 && (g_bwd_phase_mask & 1))
+  if (units > 0 && (a.phases & 1))
     delta_kernel<D><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>(P.T_q, P.Hq, static_cast<const float*>(a.o), d_o,
                                                                    a.delta);
-  if (units > 0 && (g_bwd_phase_mask & 2))
+  if (units > 0 && (a.phases & 2))
     row_kernel<D, 1><<<blocks, kWarpsPerBlock * 32, 0, a.stream>>>(dp, P.Hq, P.Hq / P.Hkv, a.pool_capacity, a.scale,
                                                                     q, k, v, nullptr, nullptr, a.lse_in, a.delta, d_o,
                                                                     static_cast<float*>(a.d_q));
   dim3 grid(P.n_pages, P.Hkv);
-  if (g_bwd_phase_mask & 4)
+  if (a.phases & 4)
     dkv_kernel<D><<<grid, kWarpsPerBlock * 32, 0, a.stream>>>(dp, P.Hq, P.Hq / P.Hkv, a.pool_capacity, a.scale, q, k, v,
                                                             a.lse_in, a.delta, d_o, static_cast<float*>(a.dk_pool),
                                                             static_cast<float*>(a.dv_pool));

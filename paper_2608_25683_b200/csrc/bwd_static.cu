@@ -22,14 +22,13 @@
 #include "kernels.h"
 #include "plan.h"
 
-struct psrl_plan {
-  psrl::Plan* p;
-};
-
 namespace {
 
-constexpr size_t kMaxDeltaFloats = size_t(4) << 20;  // n_q_heads * T_q <= 4,194,304 (16 MiB of fp32)
+// The array holds the status header, D (one float per query row and head), and - for plans whose schedule
+// splits heavy KV tiles or assembles rows from partial results - the fp32 slabs and partial dQ rows as well.
+constexpr size_t kMaxDeltaFloats = size_t(4) << 20;  // n_q_heads * T_q <= 4,194,304 (16 MiB of fp32) at most
 constexpr size_t kScratchBytes = psrl::kWsHeaderBytes + kMaxDeltaFloats * sizeof(float);
+static_assert(kScratchBytes == PSRL_BWD_STATIC_SCRATCH_BYTES, "the header states the array's size");
 
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 
@@ -60,8 +59,6 @@ void* scratch_on_current_device() {
   return g_scratch_addr[dev];
 }
 
-bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) % 16) == 0; }
-
 }  // namespace
 
 extern "C" psrl_status_t psrl_tree_attn_bwd_static(const psrl_plan_t* plan, const void* q, const void* k_pool,
@@ -72,12 +69,18 @@ extern "C" psrl_status_t psrl_tree_attn_bwd_static(const psrl_plan_t* plan, cons
   if (status_workspace) *status_workspace = nullptr;
   if (!plan || !plan->p) return PSRL_ERR_INVALID_ARG;
   const psrl::Plan& P = *plan->p;
-  if (!aligned16(q) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(o) || !aligned16(lse) ||
-      !aligned16(d_o) || !aligned16(d_q) || !aligned16(dk_pool) || !aligned16(dv_pool))
+  // the same pointer rules as psrl_tree_attn_bwd: Q-shaped tensors of a plan without query rows may be NULL
+  using psrl::ptr_aligned;
+  using psrl::ptr_aligned_q;
+  if (!ptr_aligned_q(q, 16, P) || !ptr_aligned(k_pool, 16) || !ptr_aligned(v_pool, 16) || !ptr_aligned_q(o, 16, P) ||
+      !ptr_aligned_q(lse, 16, P) || !ptr_aligned_q(d_o, 16, P) || !ptr_aligned_q(d_q, 16, P) ||
+      !ptr_aligned(dk_pool, 16) || !ptr_aligned(dv_pool, 16))
     return PSRL_ERR_INVALID_ARG;
   if (pool_capacity < P.pool_slots) return PSRL_ERR_SHAPE;
   if (!P.dev) return PSRL_ERR_WORKSPACE;  // plan not uploaded
-  // the built-in scratch is a fixed size: larger problems must use psrl_tree_attn_bwd
+  // the built-in scratch is a fixed size: a plan fits when the workspace the regular backward would ask for
+  // (psrl_bwd_workspace_bytes: header + D + split slabs + partial dQ rows) fits; larger ones must use
+  // psrl_tree_attn_bwd
   if (size_t(P.Hq) * size_t(P.T_q) > kMaxDeltaFloats) return PSRL_ERR_WORKSPACE;
   if (psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P) + psrl::ws_slab_bytes(P) + psrl::ws_part_bytes(P) > kScratchBytes)
     return PSRL_ERR_WORKSPACE;

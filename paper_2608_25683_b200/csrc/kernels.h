@@ -48,7 +48,13 @@ struct AttnArgs {
   int64_t pool_capacity;
   float scale;
   cudaStream_t stream;
+  int phases = 7;  // backward kernels to launch: bit 0 D pre-pass, bit 1 dQ, bit 2 dK/dV (7 everywhere but in benchmarks)
 };
+
+// Pointer checks of the entry points: non-NULL and aligned; Q-shaped tensors of a plan without any
+// query row are empty, so NULL is accepted for them.
+inline bool ptr_aligned(const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline bool ptr_aligned_q(const void* p, size_t a, const Plan& P) { return (P.T_q == 0 && !p) || ptr_aligned(p, a); }
 
 // fp32 SIMT path (exact-arithmetic parity path; head_dim 64 or 128)
 cudaError_t fwd_f32(const AttnArgs& a);
@@ -75,8 +81,5 @@ inline cudaError_t ensure_dynamic_smem(Kernel kernel, size_t bytes, bool (&done)
   if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
   return e;
 }
-
-// Which backward kernels to launch (profiling aid): bit 0 delta, bit 1 dQ, bit 2 dK/dV.
-extern int g_bwd_phase_mask;
 
 }  // namespace psrl

@@ -50,9 +50,6 @@ bool ok16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 }  // namespace
 }  // namespace psrl
 
-struct psrl_plan {
-  psrl::Plan* p;
-};
 
 extern "C" {
 

@@ -133,3 +133,8 @@ struct Plan {
 psrl_status_t build_plan(const psrl_tree_desc_t& desc, Plan*& out);
 
 }  // namespace psrl
+
+// The opaque handle of the C ABI (one definition for every translation unit that takes a plan).
+struct psrl_plan {
+  psrl::Plan* p;
+};

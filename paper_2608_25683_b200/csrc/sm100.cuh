@@ -186,12 +186,35 @@ __device__ __forceinline__ void fence_proxy_async() {
 // and no timeout, so it is only used where (a) the producers cannot arrive a second time before the
 // consumer has synced on the first (their next arrival depends on an MMA that the consumer issues
 // after that sync), and (b) every producer performs all its arrivals even after it gave up on a
-// wait of its own (see named_arrive_rest in the kernels), so the consumer is never left waiting.
+// wait of its own, so the consumer is never left waiting.  A producer that gave up no longer has
+// dependency (a) to pace it, and arrivals that run ahead of the consumer would wrap the barrier's
+// count and leave a residue that no later arrival completes; so on that path it stays in step by
+// hand: the consumer publishes the step it is at (StepBeacon::at, written before the step's syncs),
+// and the producer arrives for step i only once the consumer has reached step i - or stops arriving
+// once the consumer has left its loop.  Every sync of the consumer therefore gets exactly one
+// arrival per producer thread, in bounded time, on every path.
 __device__ __forceinline__ void named_arrive(uint32_t id, uint32_t n_threads) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
 }
 __device__ __forceinline__ void named_sync(uint32_t id, uint32_t n_threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+// Where the consumer of the named barriers (the MMA-issuing warp) is: `at` = the step whose syncs it is
+// about to perform or performing (-1 before the first), `left` = 1 once it has left its loop for good.
+struct StepBeacon {
+  volatile int at;
+  volatile int left;
+};
+// Producer side, only on the path of a warp that gave up on a wait: true once the consumer has reached
+// step i (arrive for it now), false if the consumer has left its loop or the bounded wait ran out (stop
+// arriving: nobody will sync again).
+__device__ __forceinline__ bool beacon_reached(const StepBeacon* b, int i) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (b->left) return false;
+    if (b->at >= i) return true;
+    __nanosleep(64);
+  }
+  return false;
 }
 
 // ---------------------------------------------------------------- TMA

@@ -21,10 +21,48 @@ void resolve() {
 }
 }  // namespace
 
+namespace {
+// Encoded maps are kept: a tensor map is a pure function of (base, shape, pitch, box), and a training step
+// calls the library with the same tensors step after step, so in steady state no call encodes anything
+// (a forward + backward would otherwise encode ~30 maps on the host, which is what bounds the time of a
+// launch-bound small case).  Small direct-mapped table, one mutex.
+struct MapKey {
+  const void* base;
+  uint64_t cols, rows, pitch;
+  uint32_t box_rows;
+  bool operator==(const MapKey& o) const {
+    return base == o.base && cols == o.cols && rows == o.rows && pitch == o.pitch && box_rows == o.box_rows;
+  }
+};
+struct MapSlot {
+  bool used = false;
+  MapKey key{};
+  CUtensorMap map;
+};
+constexpr size_t kMapSlots = 256;
+MapSlot g_maps[kMapSlots];
+std::mutex g_maps_mu;
+size_t map_hash(const MapKey& k) {
+  uint64_t h = reinterpret_cast<uint64_t>(k.base) * 0x9E3779B97F4A7C15ull;
+  h ^= (k.rows + 0x7F4A7C15ull) * 0xBF58476D1CE4E5B9ull;
+  h ^= (k.cols * 31 + k.pitch * 17 + k.box_rows) * 0x94D049BB133111EBull;
+  return size_t((h >> 29) % kMapSlots);
+}
+}  // namespace
+
 bool make_map_bf16_2d(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t pitch_bytes,
                       uint32_t box_rows) {
   std::call_once(g_once, resolve);
   if (!g_encode) return false;
+  const MapKey key{base, cols, rows, pitch_bytes, box_rows};
+  const size_t slot = map_hash(key);
+  {
+    std::lock_guard<std::mutex> lock(g_maps_mu);
+    if (g_maps[slot].used && g_maps[slot].key == key) {
+      *map = g_maps[slot].map;
+      return true;
+    }
+  }
   cuuint64_t dims[2] = {cols, rows};
   cuuint64_t strides[1] = {pitch_bytes};
   cuuint32_t box[2] = {64, box_rows};
@@ -35,6 +73,12 @@ bool make_map_bf16_2d(CUtensorMap* map, const void* base, uint64_t cols, uint64_
   if (r != CUDA_SUCCESS) {
     set_last_cuda_error(cudaErrorInvalidValue);
     return false;
+  }
+  {
+    std::lock_guard<std::mutex> lock(g_maps_mu);
+    g_maps[slot].used = true;
+    g_maps[slot].key = key;
+    g_maps[slot].map = *map;
   }
   return true;
 }

@@ -198,3 +198,32 @@ def make_inputs(T_q: int, pool_slots: int, tok_slot, n_q_heads: int, n_kv_heads:
         keep[torch.as_tensor(np.asarray(sparse_do_rows), dtype=torch.long, device=device)] = True
         d_o[~keep] = 0
     return q, k, v, d_o
+
+
+def flatten_forest(view: dict):
+    """The unshared layout: every sample becomes a root segment of its own
+    holding copies of its tokens (what a system without prefix sharing stores).
+
+    Returns (parent, seg_len, group_block_size, tok_src, first_copy) where
+    tok_src[i] is the tree token copied to flat token i and first_copy[i] says
+    whether it is that token's first copy in canonical sample order (the copy
+    that carries the token's upstream gradient row; the others get zero).
+    """
+    parent, seg_len, gbs, src = [], [], [], []
+    for e in view["sample_end_seg"]:
+        e = int(e)
+        path = list(view["anc_list"][view["anc_off"][e]:view["anc_off"][e + 1]]) + [e]
+        L = 0
+        for c in path:
+            t0 = int(view["seg_tok_off"][c])
+            n = int(view["seg_len"][c])
+            src.append(np.arange(t0, t0 + n, dtype=np.int64))
+            L += n
+        parent.append(-1)
+        seg_len.append(L)
+        gbs.append(int(view["seg_bs"][e]))
+    tok_src = np.concatenate(src)
+    _, first_idx = np.unique(tok_src, return_index=True)
+    first_copy = np.zeros(len(tok_src), dtype=bool)
+    first_copy[first_idx] = True
+    return parent, seg_len, gbs, tok_src, first_copy

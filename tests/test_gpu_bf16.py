@@ -17,7 +17,7 @@ G_TOL = 1e-2     # relative Frobenius on dQ, dK, dV
 
 def check(lib, w, seed, pad="nan", extra_capacity=0, backward=True):
     plan = build_plan(lib, w)
-    V = plan.view
+    V = plan.oracle   # the oracle's own plan (asserted byte-equal to the library's view)
     cap = V["pool_slots"] + extra_capacity
     q, k, v, d_o = make_inputs(V["T_q"], cap, V["tok_slot"], w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, seed,
                                device="cuda", pad=pad)
@@ -155,7 +155,7 @@ def test_no_queries_at_all(lib):
     write; backward still owns the gradient pools and writes zeros to every slot of every page."""
     w = Workload("nq", [-1, 0], [200, 70], [64], 4, 2, 128, "bf16", seg_flags=[0, 2])
     plan = build_plan(lib, w)
-    V = plan.view
+    V = plan.oracle   # the oracle's own plan (asserted byte-equal to the library's view)
     assert V["T_q"] == 0
     cap = V["pool_slots"] + 64
     q = torch.zeros(0, 4, 128, dtype=torch.bfloat16, device="cuda")

@@ -14,7 +14,7 @@ TOL = 1e-5  # max-abs bound for fp32 inputs, on O, dQ, dK, dV
 
 def _check(lib, w, seed, pad="nan", extra_capacity=0):
     plan = build_plan(lib, w)
-    V = plan.view
+    V = plan.oracle   # the oracle's own plan (asserted byte-equal to the library's view)
     cap = V["pool_slots"] + extra_capacity
     q, k, v, d_o = make_inputs(V["T_q"], cap, V["tok_slot"], w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, seed,
                                device="cuda", pad=pad)

@@ -15,7 +15,7 @@ def test_scatter_gather_bit_exact(lib, dtype, d):
     w = Workload("p", [-1, 0, 0, -1, 3], [333, 200, 45, 17, 129], [64, 16], 4, 2, d, dtype,
                  free_extents=[(2048, 512), (0, 160), (512, 1024), (4096, 1024)])
     plan = build_plan(lib, w)
-    V = plan.view
+    V = plan.oracle   # the oracle's own plan (asserted byte-equal to the library's view)
     T, cap = V["T"], 6000
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     g = torch.Generator(device="cuda").manual_seed(5)
@@ -38,7 +38,7 @@ def test_scatter_gather_bit_exact(lib, dtype, d):
 def test_full_size_roundtrip_and_bandwidth(lib):
     w = make_workload("c5", 1)
     plan = build_plan(lib, w)
-    V = plan.view
+    V = plan.oracle   # the oracle's own plan (asserted byte-equal to the library's view)
     T, cap = V["T"], V["pool_slots"]
     k_tok = torch.randn(T, w.n_kv_heads, 128, device="cuda").to(torch.bfloat16)
     v_tok = torch.randn(T, w.n_kv_heads, 128, device="cuda").to(torch.bfloat16)

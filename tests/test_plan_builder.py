@@ -8,7 +8,7 @@ import pytest
 
 from oracle import oracle_plan, PlanError
 from oracle.plan import PLAN_ARRAYS, PLAN_SCALARS
-from paper_2608_25683_b200.workloads import make_workload, random_forest
+from paper_2608_25683_b200.workloads import flatten_forest, make_workload, random_forest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -128,7 +128,7 @@ def test_launch_argument_checks_need_no_gpu(lib):
 def test_flatten_forest(lib):
     w = make_workload("c3", 0, scale_len=0.05)
     plan = lib.Plan(w.parent, w.seg_len, w.group_block_size, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype)
-    parent, seg_len, gbs, src, first = lib.flatten_forest(plan.view)
+    parent, seg_len, gbs, src, first = flatten_forest(plan.view)
     V = plan.view
     assert sum(seg_len) == V["flat_tokens"] == len(src)
     assert first.sum() == V["T"]

@@ -59,7 +59,8 @@ def test_token_wise_micro_batching(lib):
         pieces, budget = microbatch_tokens(parent, seg_len, alpha, M, None if flags is None else [True] * len(parent))
         want_parent, want_len, want_mb, origin = pieces_to_forest(parent, seg_len, pieces)
         got = binding.psrl_microbatch_tokens(parent, seg_len, alpha, M, flags)
-        assert got["budget"] == budget
+        # the budget is a sum of doubles: equal to one unit in the last place; the cuts are integers: exact
+        assert abs(got["budget"] - budget) <= np.spacing(max(abs(budget), abs(got["budget"])))
         assert got["parent"].tolist() == want_parent and got["seg_len"].tolist() == want_len
         assert got["mb"].tolist() == want_mb
         assert list(zip(got["seg"].tolist(), got["begin"].tolist())) == origin

@@ -2,22 +2,33 @@
 import numpy as np
 import torch
 
-from oracle import oracle_attn
+from oracle import oracle_attn, oracle_plan
+from oracle.plan import PLAN_ARRAYS, PLAN_SCALARS
 from paper_2608_25683_b200.workloads import make_inputs
 
 
+def checked_oracle_plan(view, parent, seg_len, group_block_size, seg_flags=None, free_extents=None,
+                        seg_slot_base=None):
+    """The plan of this forest built by the ORACLE, after asserting that the library's view of its own
+    plan equals it byte for byte.  Parity tests hand this one to oracle_attn, so the checker never
+    reads an index (tok_slot, anc_list, seg_q_off ...) that the product computed."""
+    want = oracle_plan(parent, seg_len, group_block_size, seg_flags, free_extents, seg_slot_base)
+    for key in PLAN_SCALARS:
+        assert view[key] == want[key], key
+    for key in PLAN_ARRAYS:
+        assert view[key].dtype == np.int32 and want[key].dtype == np.int32, key
+        assert view[key].tobytes() == want[key].tobytes(), key
+    return want
+
+
 def build_plan(lib, w, upload=True):
+    """The library's plan of workload `w`; `plan.oracle` is the oracle's plan of the same forest."""
     plan = lib.Plan(w.parent, w.seg_len, w.group_block_size, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype,
                     w.seg_flags, w.free_extents)
+    plan.oracle = checked_oracle_plan(plan.view, w.parent, w.seg_len, w.group_block_size, w.seg_flags, w.free_extents)
     if upload:
         plan.upload()
     return plan
-
-
-def oracle_view(view):
-    """The oracle functions take the plan as a dict of numpy arrays; the C++ plan
-    is bit-identical to the oracle's (tests/test_plan_builder.py), so its view serves."""
-    return view
 
 
 def run_gpu(lib, plan, q, k, v, d_o, scale, backward=True):
