@@ -350,7 +350,6 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
     const uint32_t t_lane = tmem + (uint32_t((warp & 3) * 32) << 16);
     const f32x2 scale2 = make_f32x2(p.scale_log2, p.scale_log2);
     bool ok = true;
-    bool arrive = true;   // false once the MMA warp has left its loop: nobody syncs any more
     for (int i = 0; i < n_it; ++i) {
       int g, row0, nvq, qpos0; bool diag;
       step(i, g, row0, nvq, diag, qpos0);
@@ -405,9 +404,10 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
           quarters_sent = g + 1;
         }
       }
-      if (!ok && arrive) arrive = beacon_reached(&s_beacon, i);
-      if (arrive)
-        for (int g = quarters_sent; g < 4; ++g) named_arrive(kBarP + g, kBarThreads);   // gave up on a wait
+      if (!ok) {   // gave up on a wait: the remaining arrivals of this step, in step with the MMA warp
+        if (!beacon_reached(&s_beacon, i)) break;   // the MMA warp has left its loop: nobody syncs any more
+        for (int g = quarters_sent; g < 4; ++g) named_arrive(kBarP + g, kBarThreads);
+      }
       // ---- half-step 2: dS^T = P^T o dP^T_aug (-D is already inside) ----
       if (ok) ok = mbar_wait(&bar.dp_full, i & 1, abortp, p.status);
       if (ok) {
@@ -430,8 +430,8 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
       }
       tmem_wait_st();
       tc_fence_before();
-      if (!ok && arrive) arrive = beacon_reached(&s_beacon, i);
-      if (arrive) named_arrive(kBarDs, kBarThreads);
+      if (!ok && !beacon_reached(&s_beacon, i)) break;
+      named_arrive(kBarDs, kBarThreads);
     }
     // ---- epilogue: warps 0-3 take dV, warps 4-7 take dK ----
     if (ok && n_it > 0) ok = mbar_wait(&bar.acc_full, 0, abortp, p.status);

@@ -78,7 +78,6 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
   __shared__ Barriers bar;
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
-  __shared__ StepBeacon s_beacon;   // the MMA warp's position, for softmax warps that gave up on a wait
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // ---- which work item ----
@@ -93,8 +92,6 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
 
   if (tid == 0) {
     s_abort = 0;
-    s_beacon.at = -1;
-    s_beacon.left = 0;
     mbar_init(&bar.q_full, 1);
     for (int i = 0; i < KS; ++i) { mbar_init(&bar.k_full[i], 1); mbar_init(&bar.k_empty[i], 1); }
     for (int i = 0; i < VS; ++i) { mbar_init(&bar.v_full[i], 1); mbar_init(&bar.v_empty[i], 1); }
@@ -190,7 +187,6 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       }
       for (int j = 0; ok && j < n_tiles; ++j) {
         const int vs = j % VS;
-        if (lane == 0) s_beacon.at = j;   // before this tile's syncs (read only by warps that gave up)
         for (int q = 0; ok && q < nq; ++q) {
           // one round of barrier tests per head: for head 0 also the V tile of this step and the K tile
           // of the next one (each separate wait would cost the issuing warp hundreds of cycles)
@@ -217,7 +213,6 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
           }
         }
       }
-      if (lane == 0) s_beacon.left = 1;   // no sync follows on any path
     }
   } else if (warp < 4 * nq) {
     // ======================= softmax warpgroups =======================
@@ -231,7 +226,6 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
     float m_ref = -CUDART_INF_F, l_run = 0.f;
     const f32x2 scale2 = make_f32x2(p.scale_log2, p.scale_log2);
     bool ok = true;
-    bool arrive = true;   // false once the MMA warp has left its loop: nobody syncs any more
     int nv_next = path_nvalid[0];
     for (int j = 0; j < n_tiles; ++j) {
       const int n_valid = nv_next;
@@ -241,7 +235,10 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       const bool need_mask = diag || n_valid < 128;
       // A warp that gave up on a wait (ok == false) skips the tile's work but still arrives on the named
       // barrier of every remaining tile, so that the MMA warp is never left waiting at one - one arrival
-      // per tile, and for tile j only once the MMA warp has reached tile j (see StepBeacon).
+      // per tile, and for tile j only once the MMA warp has synced on tile j-1: that is what a completed
+      // o_full[q] phase j-1 says (its commit follows P V(j-1), issued right behind that sync).  The MMA
+      // warp therefore carries nothing for this path (a shared-memory store per tile in that warp cost the
+      // kernel 1.5-3 %).  If the phase never completes the MMA warp has left its loop: stop arriving.
       do {
       if (!ok) break;
       // ---- softmax of this tile: the whole score row in one round trip to tensor memory ----
@@ -356,8 +353,8 @@ fwd_kernel(const __grid_constant__ FwdMaps maps, const FwdParams p) {
       tmem_wait_st();
       } while (false);
       tc_fence_before();
-      if (!ok && arrive) arrive = beacon_reached(&s_beacon, j);
-      if (arrive) named_arrive(kBarP + q, kBarThreads);
+      if (!ok && j > 0 && !mbar_wait_bounded(&bar.o_full[q], (j - 1) & 1)) break;
+      named_arrive(kBarP + q, kBarThreads);
     }
     // ---- last tile's product, normalise, store ----
     if (ok) ok = mbar_wait(&bar.o_full[q], (n_tiles - 1) & 1, abortp, p.status);

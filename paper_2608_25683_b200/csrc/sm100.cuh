@@ -61,6 +61,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
+// Bounded wait that ignores the abort flag (used only on the path of a warp that has already given up and
+// has to learn how far the MMA-issuing warp got before it arrives on a named barrier for it).
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    if (it > 64) __nanosleep(64);
+  }
+  return false;
+}
+
 // Bounded wait of a TMA producer thread on a ring stage.  The producer is usually ahead and
 // spends most of its time here; it sleeps between polls so that it takes no issue slots from the
 // softmax warps of its SM sub-partition.
@@ -189,10 +199,11 @@ __device__ __forceinline__ void fence_proxy_async() {
 // wait of its own, so the consumer is never left waiting.  A producer that gave up no longer has
 // dependency (a) to pace it, and arrivals that run ahead of the consumer would wrap the barrier's
 // count and leave a residue that no later arrival completes; so on that path it stays in step by
-// hand: the consumer publishes the step it is at (StepBeacon::at, written before the step's syncs),
-// and the producer arrives for step i only once the consumer has reached step i - or stops arriving
-// once the consumer has left its loop.  Every sync of the consumer therefore gets exactly one
-// arrival per producer thread, in bounded time, on every path.
+// hand: it arrives for step i only once it knows that the consumer has synced on step i-1 - from a
+// step counter the consumer publishes (StepBeacon, dK/dV kernel) or from an mbarrier phase that the
+// consumer's MMAs of step i-1 complete (forward) - and stops arriving once the consumer has left its
+// loop.  Every sync of the consumer therefore gets exactly one arrival per producer thread, in
+// bounded time, on every path.
 __device__ __forceinline__ void named_arrive(uint32_t id, uint32_t n_threads) {
   asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
 }

@@ -191,14 +191,32 @@ def test_many_short_branches_nested(lib):
     assert S["H"]["n_merge_rows"] > 0
 
 
-def test_benchmark_trees_are_not_cascaded(lib):
-    """Branches of hundreds of tokens fill their own tiles: no packed items, no merge."""
-    for name in ("c2", "c3"):
-        w = make_workload(name, 7)
-        plan = binding.Plan(w.parent, w.seg_len, w.group_block_size, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype)
-        S = decode(plan)
-        assert S["H"]["n_merge_rows"] == 0 and S["H"]["n_part_rows"] == 0
-        assert all(q[6] == 1 and q[7] == -1 for q in S["qt"].tolist())
+def test_which_benchmark_trees_are_cascaded(lib):
+    """c2, c3, c5: branches of hundreds or thousands of tokens fill their own tiles - no packed items, no
+    merge.  c4 mixes long prefixes with suffixes down to 64 tokens: some of its groups are cascaded, so its
+    forward and dQ are followed by the merge kernels; every merged row then has at least two parts and every
+    partial row belongs to exactly one merged row."""
+    for name in ("c2", "c3", "c5"):
+        for seed in (7, 2000):
+            w = make_workload(name, seed)
+            plan = binding.Plan(w.parent, w.seg_len, w.group_block_size, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype)
+            S = decode(plan)
+            assert S["H"]["n_merge_rows"] == 0 and S["H"]["n_part_rows"] == 0
+            assert all(q[6] == 1 and q[7] == -1 for q in S["qt"].tolist())
+            assert binding.psrl_launch_count(plan, False) == 1
+    w = make_workload("c4", 2000)
+    plan = binding.Plan(w.parent, w.seg_len, w.group_block_size, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype,
+                        w.seg_flags, w.free_extents)
+    S = decode(plan)
+    H = S["H"]
+    assert H["n_merge_rows"] > 0 and binding.psrl_launch_count(plan, False) == 2
+    off = S["merge_off"]
+    assert (np.diff(off) >= 2).all()
+    parts = np.sort(S["merge_parts"])
+    assert len(parts) == H["n_part_rows"] and (parts == np.arange(H["n_part_rows"])).all()
+    # every work item of every kernel has at least one step wherever its kernel syncs on a named barrier
+    assert all(q[5] >= 1 for q in S["qt"].tolist())
+    assert all(k[6] > k[5] for k in S["kvi"].tolist())
 
 
 def test_random_forests(lib):
