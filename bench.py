@@ -36,8 +36,9 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel
 # (dkv_kernel), from the ncu captures summarised under profiles/ ; None = not captured.
-NCU_TRAFFIC_BYTES = {"c2": 355363584 + 24176640,   # profiles/dkv_kernel_c2.md
-                     "c3": 1886000000 + 72000000}   # profiles/kernels_c3.md
+NCU_TRAFFIC_BYTES = {"c2": 353620000 + 24440000,       # profiles/dkv_kernel_c2.md
+                     "c3": 1886000000 + 72000000,      # profiles/kernels_c3.md
+                     "c5": 208710000000 + 836200000}   # profiles/dkv_kernel_c5_dram.md (full size, one pass)
 
 
 def peaks():
