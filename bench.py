@@ -691,7 +691,8 @@ def measure_config(args, lib, name, device, rank, world, local, headline):
     ridge = pk["bf16_tflops"] * 1e12 / (pk["hbm_gbs"] * 1e9)
     hbm_bound = w.dtype == "bf16" and flops / step_bytes < ridge
     timing_note = ("each kernel timed inside running steps (events between the step's parts), mean of %d steps, "
-                   "SM clock sampled over those steps" % n_ph)
+                   "SM clock sampled over those steps; in a whole step of a small plan dQ and dK/dV run side by "
+                   "side on two streams, so there the parts add up to more than the step" % n_ph)
     if hbm_bound:
         achieved = kbytes[dom] / (kern[dom] * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
@@ -928,7 +929,7 @@ def main():
                 dtype=res["dtype"], data="synthetic", config=res["config"], clocks=res["clocks"], e2e=res["e2e"],
                 gpu_launches=res["gpu_launches"], roofline=res["roofline"], cpu_baseline=cpu, step_ms=res["step_ms"],
                 bitwise_reproducible_3_runs=res["bitwise_reproducible_3_runs"], plan=res["plan"],
-                unshared=res["unshared"], frac_of_bf16_peak=res["frac_of_bf16_peak"],
+                unshared=res["unshared"], cuda_graph=res.get("cuda_graph"), frac_of_bf16_peak=res["frac_of_bf16_peak"],
                 per_config=per_config or None, library_context=extra.get("library_context"),
                 microbatch=extra.get("microbatch"), schedule=extra.get("schedule"), kv_pack=extra.get("kv_pack"))
     print(json.dumps(line), flush=True)

@@ -96,6 +96,7 @@ extern "C" psrl_status_t psrl_tree_attn_bwd_static(const psrl_plan_t* plan, cons
   a.slabs = reinterpret_cast<float*>(ws + psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P));
   a.part = reinterpret_cast<float*>(ws + psrl::kWsHeaderBytes + psrl::ws_delta_bytes(P) + psrl::ws_slab_bytes(P));
   a.pool_capacity = pool_capacity; a.scale = softmax_scale; a.stream = static_cast<cudaStream_t>(stream);
+  a.fork = false;   // no side stream here: creating one is a resource allocation this entry point promises not to make
   // the array keeps the previous call's contents: the status header must start at zero;
   // D is fully rewritten by the pre-pass before anything reads it
   cudaError_t e = cudaMemsetAsync(ws, 0, psrl::kWsHeaderBytes, a.stream);

@@ -49,6 +49,7 @@ struct AttnArgs {
   float scale;
   cudaStream_t stream;
   int phases = 7;  // backward kernels to launch: bit 0 D pre-pass, bit 1 dQ, bit 2 dK/dV (7 everywhere but in benchmarks)
+  bool fork = true;  // bf16 backward: dK/dV on an internal side stream beside dQ (false: everything on `stream`)
 };
 
 // Pointer checks of the entry points: non-NULL and aligned; Q-shaped tensors of a plan without any
