@@ -79,6 +79,31 @@ __device__ __forceinline__ void zero_tile_row(uint8_t* tile, int row) {
   }
 }
 
+// Block order of the three main kernels: block b -> (work item, unit u of the item; u = KV head, query head or
+// head pair).  chunk == 0: item-major (b = item * per_item + u), which keeps the longest-first order of the items
+// exact - used for small launches, where that order is what balances the SMs.  chunk > 0 (large launches):
+// unit-major inside chunks of `chunk` items, so that the CTAs that run at the same time mostly share one KV head:
+// they then stream the same K/V tiles (forward, dQ) or the Q and dO rows of the same query heads (dK/dV), which
+// compete for the L2 with a quarter or an eighth of the whole set.  The chunks still follow the longest-first order.
+__device__ __forceinline__ void block_to_item(int b, int n_items, int per_item, int chunk, int& item, int& u) {
+  if (chunk > 0) {
+    const int per = chunk * per_item;
+    const int c = b / per, r = b % per;
+    const int in_chunk = min(chunk, n_items - c * chunk);
+    u = r / in_chunk;
+    item = c * chunk + r % in_chunk;
+  } else {
+    item = b / per_item;
+    u = b % per_item;
+  }
+}
+// Items per chunk for a launch of n_items work items on a device with n_sm SMs (0 = item-major): chunks of
+// one item per SM once the launch has at least `min_waves` items per SM (measured: dK/dV gains from one wave
+// on, -3 % on the 276-item tree configuration and -6 % on the large ones; dQ only on the large ones, -2 %).
+inline int block_order_chunk(int64_t n_items, int n_sm, int min_waves) {
+  return n_items >= int64_t(min_waves) * n_sm ? n_sm : 0;
+}
+
 bool make_pool_maps(PoolMaps* maps, const void* k_pool, const void* v_pool, int Hkv, int64_t cap);
 
 }  // namespace psrl

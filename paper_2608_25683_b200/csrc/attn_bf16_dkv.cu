@@ -53,6 +53,7 @@ struct Params {
   const int32_t* blob;
   int32_t off_kvi, off_kvt, off_page_slot, off_split;
   int32_t Hq, Hkv, G, T_q;
+  int32_t chunk;   // items per KV-head-major chunk of the block order, 0 = item-major
   int64_t cap;
   float scale, scale_log2, inv_scale;
   const float* lse;
@@ -125,7 +126,13 @@ dkv_kernel(const __grid_constant__ Maps maps, const Params p) {
   __shared__ StepBeacon s_beacon;   // the MMA warp's position, for softmax warps that gave up on a wait
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int item = blockIdx.x / p.Hkv, hk = blockIdx.x % p.Hkv;
+  // Block order.  Small launches: item-major (block = item x Hkv + hk), which keeps the longest-first order of
+  // the items exact.  Large launches: KV-head-major inside chunks of `p.chunk` items, so that the CTAs that run
+  // at the same time mostly belong to one KV head and the Q and dO rows they stream (those of that head's query
+  // heads) compete for the L2 with a quarter or an eighth of the set; the chunks still follow the longest-first
+  // order.
+  int item, hk;
+  block_to_item(int(blockIdx.x), int(gridDim.x) / p.Hkv, p.Hkv, p.chunk, item, hk);
   const KvItem it = reinterpret_cast<const KvItem*>(p.blob + p.off_kvi)[item];
   const KvTile kt = reinterpret_cast<const KvTile*>(p.blob + p.off_kvt)[it.kvt];
   const int n_own_sub = it.own_q_row0 >= 0 ? (it.own_q_end - it.own_q_row0 + kSubRows - 1) / kSubRows : 0;
@@ -565,6 +572,7 @@ psrl_status_t dkv_bf16(const AttnArgs& a) {
   p.lse = a.lse_in; p.delta = a.delta; p.slabs = a.slabs;
   p.dk = static_cast<__nv_bfloat16*>(a.dk_pool); p.dv = static_cast<__nv_bfloat16*>(a.dv_pool);
   p.status = a.status;
+  p.chunk = block_order_chunk(int64_t(P.kv_items.size()), resident_ctas(), 1);
   const int64_t grid = int64_t(P.kv_items.size()) * P.Hkv;
   if (grid > INT32_MAX) return PSRL_ERR_SHAPE;
   dkv_kernel<<<unsigned(grid), kThreads, smem, a.stream>>>(m, p);

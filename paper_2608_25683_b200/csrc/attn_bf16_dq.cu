@@ -45,6 +45,7 @@ struct Params {
   const int32_t* blob;
   int32_t off_qt, off_kvt, off_path_tiles, off_path_nvalid, off_path_loads, off_page_slot;
   int32_t Hq, G, T_q;
+  int32_t chunk;   // block order, see block_to_item
   int64_t cap;
   float scale, scale_log2;
   const float* lse;
@@ -73,7 +74,9 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
   __shared__ int s_abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int item = blockIdx.x / p.Hq, h = blockIdx.x % p.Hq, hk = h / p.G;
+  int item, h;
+  block_to_item(int(blockIdx.x), int(gridDim.x) / p.Hq, p.Hq, p.chunk, item, h);
+  const int hk = h / p.G;
   const QTile qt = reinterpret_cast<const QTile*>(p.blob + p.off_qt)[item];
   const int32_t* path_nvalid = p.blob + p.off_path_nvalid + qt.pt_begin;
   const int n_tiles = qt.n_kv_tiles;
@@ -121,7 +124,9 @@ dq_kernel(const __grid_constant__ Maps maps, const Params p) {
       // order, one per SM): its Q and dO tiles go to the L2 now, so that its first step does not wait for HBM.
       const int nb = atomicAdd(p.done_ctr, 1) + p.resident;
       if (nb < int(gridDim.x)) {
-        const int nrow = reinterpret_cast<const QTile*>(p.blob + p.off_qt)[nb / p.Hq].q_row0, nh = nb % p.Hq;
+        int nitem, nh;
+        block_to_item(nb, int(gridDim.x) / p.Hq, p.Hq, p.chunk, nitem, nh);
+        const int nrow = reinterpret_cast<const QTile*>(p.blob + p.off_qt)[nitem].q_row0;
         tma_prefetch_2d(&maps.q, nh * 128, nrow);
         tma_prefetch_2d(&maps.q, nh * 128 + 64, nrow);
         tma_prefetch_2d(&maps.d_o, nh * 128, nrow);
@@ -369,6 +374,7 @@ psrl_status_t dq_bf16(const AttnArgs& a) {
   p.lse = a.lse_in; p.delta = a.delta; p.d_q = static_cast<__nv_bfloat16*>(a.d_q); p.status = a.status;
   p.part = a.part;
   p.done_ctr = a.status + kWsCtrDq; p.resident = resident_ctas();
+  p.chunk = block_order_chunk(int64_t(P.q_tiles.size()), p.resident, 4);
   const int64_t grid = int64_t(P.q_tiles.size()) * P.Hq;
   if (grid > INT32_MAX) return PSRL_ERR_SHAPE;
   dq_kernel<<<unsigned(grid), kThreads, smem, a.stream>>>(m, p);
