@@ -37,8 +37,8 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel
 # (dkv_kernel), from the ncu captures summarised under profiles/ ; None = not captured.
 NCU_TRAFFIC_BYTES = {"c2": 353620000 + 24440000,       # profiles/dkv_kernel_c2.md
-                     "c3": 1886000000 + 72000000,      # profiles/kernels_c3.md
-                     "c5": 208710000000 + 836200000}   # profiles/dkv_kernel_c5_dram.md (full size, one pass)
+                     "c3": 1140000000 + 65560000,      # profiles/dram_traffic_c5_c3.md
+                     "c5": 92590000000 + 835340000}    # profiles/dram_traffic_c5_c3.md (full size, one pass)
 
 
 def peaks():
