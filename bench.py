@@ -7,8 +7,8 @@ mask counts, no tile padding, no duplicated prefix work, no recompute).
 
   python bench.py --gpus N --steps K --warmup W [--config c2] [--impl reference]
 
-Without --config the headline is c5 (the largest single-GPU configuration) and c2, c3, c4
-and the HBM-bound c2s are measured in the same run and reported under `per_config`.
+Without --config the headline is c5 (the largest single-GPU configuration) and c1 (fp32), c2, c3, c4
+and the small-suffix case c2s are measured in the same run and reported under `per_config`.
 
 One step = one pass of the whole hot path (forward, D pre-pass, dQ, dK/dV) over
 one synthetic batch.  N > 1 (torchrun): every rank runs an independent batch
@@ -714,7 +714,13 @@ def measure_config(args, lib, name, device, rank, world, local, headline):
     roofline.update(kernel_timing=timing_note, kernel_clocks=kclk, sum_kernel_ms=round(sum_ms, 4),
                     sum_kernel_ms_over_step_ms=round(sum_ms / ms, 4))
     if w.dtype != "bf16":
-        roofline["bound"] = "alu"
+        # fp32 SIMT path: plain FMA arithmetic.  Peak from the unit counts and the clock: 148 SMs x 128 fp32 lanes
+        # x 2 flop x 1.965 GHz = 74.4 TFLOP/s (the path keeps its long sums in fp64, which runs far below that:
+        # the figure is a ceiling, and the configuration it serves is launch-bound)
+        alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        roofline.update(bound="alu", peak=round(alu_peak, 1), frac=round(achieved / alu_peak, 6),
+                        peak_source="derived: 148 SMs x 128 fp32 lanes x 2 flop x 1.965 GHz")
+        roofline.pop("frac_of_sustained", None)
 
     # ---- end to end through the public call with host buffers ----
     hq, hk, hv, hdo = (x.cpu().pin_memory() for x in (r.q, r.k, r.v, r.d_o))
@@ -857,7 +863,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default=None,
                     help="one configuration (c1..c5, c2s).  Default: c5 is the headline (the largest single-GPU "
-                         "configuration) and c2, c3, c4 and the HBM-bound c2s are measured too, under per_config")
+                         "configuration) and c1 (fp32), c2, c3, c4 and the small-suffix c2s are measured too, under per_config")
     ap.add_argument("--seed", type=int, default=2000)
     ap.add_argument("--cpu-samples", type=int, default=4, help="samples in the oracle's timed sample")
     ap.add_argument("--ref-samples", type=int, default=2, help="samples per step of --impl reference")
@@ -876,7 +882,7 @@ def main():
                     help="also run the group as one micro-batch per branch with the Dynamic Block Caching manager")
     args = ap.parse_args()
     head_name = args.config or "c5"
-    others = [] if args.config else ["c2", "c3", "c4", "c2s"]
+    others = [] if args.config else ["c1", "c2", "c3", "c4", "c2s"]
     if args.impl == "reference":
         args.config = head_name
         run_reference(args)
