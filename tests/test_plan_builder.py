@@ -195,3 +195,19 @@ def test_adaptive_blocks_bit_exact(lib):
     with pytest.raises(lib.PsrlError) as e:     # adaptive blocks exist on the tensor-core path only
         lib.Plan([-1], [40], [0], 2, 2, 64, "f32")
     assert e.value.name == "PSRL_ERR_UNSUPPORTED"
+
+
+def test_static_backward_limit_is_the_whole_workspace(lib):
+    """The built-in scratch array of psrl_tree_attn_bwd_static stands in for the whole backward workspace: the
+    header's constant equals the binding's, a plan under the D limit can still be over the array's size once the
+    slabs of its split KV tiles are counted (c3), and small plans fit."""
+    src = open(os.path.join(ROOT, "include", "psrl.h")).read()
+    m = re.search(r"#define PSRL_BWD_STATIC_SCRATCH_BYTES \(\(size_t\)(\d+)\)", src)
+    assert m and int(m.group(1)) == lib.BWD_STATIC_SCRATCH_BYTES == 16 * 1024 * 1024 + 256
+    w = make_workload("c3", 2000)
+    plan = lib.Plan(w.parent, w.seg_len, w.group_block_size, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype)
+    assert plan.view["T_q"] * w.n_q_heads < 4 * 1024 * 1024
+    assert plan.bwd_workspace_bytes() > lib.BWD_STATIC_SCRATCH_BYTES
+    w = make_workload("c2", 2000)
+    plan = lib.Plan(w.parent, w.seg_len, w.group_block_size, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype)
+    assert plan.bwd_workspace_bytes() <= lib.BWD_STATIC_SCRATCH_BYTES
