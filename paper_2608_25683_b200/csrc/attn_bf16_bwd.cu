@@ -35,11 +35,12 @@ struct SideStream {
   bool ok = false;
 };
 SideStream g_side[64];
-std::mutex g_side_mu;
+std::mutex g_side_mu;        // serialises the fork / join enqueue sequences of a device
+std::mutex g_side_create_mu; // guards the one-time creation
 SideStream* side_stream() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  std::lock_guard<std::mutex> lock(g_side_mu);
+  std::lock_guard<std::mutex> lock(g_side_create_mu);
   SideStream& s = g_side[dev];
   if (!s.ok) {
     if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
@@ -104,6 +105,9 @@ psrl_status_t bwd_bf16(const AttnArgs& a) {
   SideStream* side = (a.fork && small && (a.phases & 6) == 6) ? side_stream() : nullptr;
   if (side) {
     // ---- dK, dV on the side stream, dQ on the caller's; join ----
+    // The two events are shared by every call on the device: the whole record / wait sequence is enqueued under
+    // the lock, so that calls from several host threads cannot pair one call's wait with another call's record.
+    std::lock_guard<std::mutex> lock(g_side_mu);
     cudaError_t e = cudaEventRecord(side->fork, a.stream);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(side->stream, side->fork, 0);
     if (e != cudaSuccess) { set_last_cuda_error(e); return PSRL_ERR_CUDA; }
